@@ -23,9 +23,14 @@ What is defined here (paper sections in brackets):
   tiny inputs to show that it agrees with `standalone_attend` (the paper's
   equivalence claim) and that the structural attended set equals the predicates.
 
+* `tuple_inputs`, `attend_tuple` -- assemble the standalone prompt of one (prompt,
+  question, step, layer, KV head) from a workload's raw accessors and evaluate it.
+  Pinned by: the dense formulation over a stacked sequence assembled independently
+  in the tests, with the KV head of each query head chosen by an explicit repeat.
+
 Numeric attention values: parity unpinned by the paper (it prints no attention
-value); they are pinned by the library routine, closed forms and invariants named
-above, in tests/test_oracle_*.py.
+value); every function here is pinned by the library routine, closed forms and
+invariants named above, in tests/test_oracle_pins.py.
 """
 from __future__ import annotations
 
@@ -186,14 +191,15 @@ def dense_attend(q_raw, k_raw, v_raw, pos, mask, theta: float) -> np.ndarray:
 
 
 # --------------------------------------------------------------------------- per-tuple driver
-def attend_tuple(wl, b: int, k: int, s: int, layer: int, kv_head: int, ctx_cache: dict | None = None,
-                 step_cache: dict | None = None) -> np.ndarray:
-    """Oracle output for question k (global id) of prompt b at decode step s, one layer,
-    all query heads of one KV head: [G, D] fp64.
+def tuple_inputs(wl, b: int, k: int, s: int, layer: int, kv_head: int, ctx_cache: dict | None = None,
+                 step_cache: dict | None = None):
+    """Raw tensors of the standalone prompt of question k (global id) of prompt b at decode step s, one layer, one KV
+    head: (k_raw [T, D], v_raw [T, D], q_raw [G, D]) in fp64, T = L_b + n_k + s + 1.
 
-    `wl` is any object with the raw-tensor accessors of a workload (ctx_kv,
-    question_kv, step_kv, step_q, geom); this function only concatenates the
-    standalone prompt's tokens and calls `standalone_attend`.
+    The prompt is the context tokens, the question's tokens, then the answer tokens fed at steps 0..s (the last one is
+    the token whose query is evaluated; Sec. 3, Sec. 4.2).  The G query heads [kv_head*G, (kv_head+1)*G) share KV head
+    `kv_head`.  `wl` is any object with the raw-tensor accessors of a workload (ctx_kv, question_kv, step_kv, step_q,
+    geom); the caches only avoid regenerating the same raw tensors.
     """
     g = wl.geom
     G = g.n_q_heads // g.n_kv_heads
@@ -220,4 +226,13 @@ def attend_tuple(wl, b: int, k: int, s: int, layer: int, kv_head: int, ctx_cache
         ks.append(ka[None, kv_head].double().numpy())
         vs.append(va[None, kv_head].double().numpy())
     q = wl.step_q(s, layer, [k])[0, kv_head * G:(kv_head + 1) * G].double().numpy()
-    return standalone_attend(np.concatenate(ks), np.concatenate(vs), q, g.rope_theta)
+    return np.concatenate(ks), np.concatenate(vs), q
+
+
+def attend_tuple(wl, b: int, k: int, s: int, layer: int, kv_head: int, ctx_cache: dict | None = None,
+                 step_cache: dict | None = None) -> np.ndarray:
+    """Oracle output for question k (global id) of prompt b at decode step s, one layer, all query heads of one KV
+    head: [G, D] fp64 -- `standalone_attend` on the standalone prompt assembled by `tuple_inputs`.  Pinned by the
+    dense-mask formulation assembled independently in the tests (the equivalence of Sec. 4.2)."""
+    k_raw, v_raw, q_raw = tuple_inputs(wl, b, k, s, layer, kv_head, ctx_cache, step_cache)
+    return standalone_attend(k_raw, v_raw, q_raw, wl.geom.rope_theta)

@@ -236,3 +236,73 @@ def test_answers_do_not_depend_on_question_order_or_duplicates():
     pw = Permuted()
     for newk, oldk in enumerate(pw.order):
         np.testing.assert_array_equal(orc.attend_tuple(pw, 0, newk, 1, 0, 1), outs[oldk])
+
+
+# ------------------------------------------------------------------ the per-tuple driver
+def _dense_rows_of_step(wl, b, s, layer):
+    """Dense-mask formulation of prompt b at decode step s: for every query head, the rows of the answer tokens fed at
+    step s, computed by dense_attend over the whole stacked sequence.  The stacked sequence is assembled here from the
+    workload's raw accessors, independently of attend_tuple; the KV head of a query head is chosen by an explicit
+    repeat of every KV head G times (the order of HF `repeat_kv`: query heads [g*G, (g+1)*G) share KV head g)."""
+    g = wl.geom
+    G = g.n_q_heads // g.n_kv_heads
+    L = int(wl.ctx_len[b])
+    k0, k1 = int(wl.q_begin[b]), int(wl.q_begin[b + 1])
+    q_lens = [int(wl.q_len[k]) for k in range(k0, k1)]
+    # answer tokens in the cache after the append of step s: a question with stop step e has fed min(e, s + 1) tokens
+    n_answer = [min(int(wl.stop[k]), s + 1) for k in range(k0, k1)]
+    pos, ctx, qtn, tag = orc.stacked_sequence(0, [L], [q_lens], [n_answer])
+    mask = orc.dense_mask(pos, ctx, qtn)
+    n = len(pos)
+    kc, vc = wl.ctx_kv(b, layer)
+    K = np.zeros((n, g.n_kv_heads, g.head_dim))
+    V = np.zeros_like(K)
+    Q = np.zeros((n, g.n_q_heads, g.head_dim))
+    rows = {}
+    for i, (kind, _, kk, idx) in enumerate(tag):
+        k = k0 + kk
+        if kind == "c":
+            K[i], V[i] = kc[idx].double().numpy(), vc[idx].double().numpy()
+        elif kind == "x":
+            kq, vq = wl.question_kv(k, layer)
+            K[i], V[i] = kq[idx].double().numpy(), vq[idx].double().numpy()
+        else:
+            ka, va = wl.step_kv(idx, layer, [k])
+            K[i], V[i] = ka[0].double().numpy(), va[0].double().numpy()
+            if idx == s:
+                Q[i] = wl.step_q(s, layer, [k])[0].double().numpy()
+                rows[k] = i
+    K_rep, V_rep = np.repeat(K, G, axis=1), np.repeat(V, G, axis=1)  # [n, Hq, D]
+    out = {}
+    for h in range(g.n_q_heads):
+        o = orc.dense_attend(Q[:, h], K_rep[:, h], V_rep[:, h], pos, mask, g.rope_theta)
+        for k, i in rows.items():
+            out[(k, h)] = o[i]
+    return out
+
+
+def test_attend_tuple_equals_the_dense_mask_formulation():
+    # Sec. 4.2: the IPPD output of an answer token under the dense mask over the stacked sequence equals the output of
+    # its triplet prompted alone.  attend_tuple assembles the standalone prompt; the dense side is assembled above from
+    # the raw accessors without it.  Two prompts, G = 2 and G = 4, ragged question lengths and stop steps, steps >= 2:
+    # a wrong number of answer tokens (range(s) for range(s + 1)), a KV-head slice shifted by one query head, a wrong
+    # question's tokens or a wrong step's query each break the agreement.
+    from paper_2609_05707_b200 import workloads as W
+    for hq, hkv in [(4, 2), (8, 2)]:
+        wl = W.custom_workload("pin", W.Geometry(2, hq, hkv, 16, 1e4), 77, [9, 5], [3, 2], [2, 4, 1, 3, 2],
+                               [4, 1, 3, 2, 4])
+        G = hq // hkv
+        checked = 0
+        for s in range(wl.n_steps):
+            act = wl.active(s)
+            for b in range(wl.n_prompts):
+                dense = _dense_rows_of_step(wl, b, s, layer=1)
+                mine = [int(k) for k in act if wl.prompt_of[k] == b]
+                assert sorted({k for k, _ in dense}) == mine  # exactly the active questions have a row at step s
+                for k in mine:
+                    for kv_head in range(hkv):
+                        got = orc.attend_tuple(wl, b, k, s, 1, kv_head)
+                        for j in range(G):
+                            np.testing.assert_allclose(got[j], dense[(k, kv_head * G + j)], atol=1e-12, rtol=0)
+                            checked += 1
+        assert checked == int(wl.stop.sum()) * hq
