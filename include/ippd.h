@@ -138,19 +138,30 @@ int ippd_set_option(ippd_layout_t* layout, int32_t key, int64_t value);
  * finished answers are no longer appended).  active_q[A]: strictly increasing
  * global question ids (host).  answer_idx[A]: the step index s of each (host);
  * the token fed is answer token y_{s+1} at virtual position L_b + n_k + s.
- * Builds the split-KV work list on the host and enqueues ONE small host-to-device
- * copy on `stream`; the following ippd_append_kv(STEP) / ippd_decode_attention
- * calls on the same stream use it for every layer.  A == 0 is allowed (the step
- * is then empty).  Errors: IPPD_ERR_INVALID_ARG, IPPD_ERR_CAPACITY (answer_idx >=
- * max_new), IPPD_ERR_NOT_BOUND, IPPD_ERR_CUDA.
+ * Builds the step's work list (row blocks, key tiles, packed branch pieces) on the
+ * host and stages it in a pinned slot; nothing is enqueued here.  The first
+ * ippd_append_kv(STEP) / ippd_decode_attention call that follows moves the
+ * descriptor to the device on ITS stream (inside its own kernel where it can), and
+ * every later call of the step, for any layer, reuses it.  `stream` is only
+ * remembered as the stream ippd_poll_status waits on.  A == 0 is allowed (the step
+ * is then empty).  The descriptor always fits its staging slot for any step the
+ * layout admits (see ippd_step_descriptor_bytes).  Errors: IPPD_ERR_INVALID_ARG,
+ * IPPD_ERR_CAPACITY (answer_idx >= max_new), IPPD_ERR_NOT_BOUND, IPPD_ERR_CUDA.
  */
 int ippd_begin_step(ippd_layout_t* layout, const int32_t* active_q, const int32_t* answer_idx,
                     int32_t n_active, void* stream);
 
+/* Host-only: the size in bytes of the descriptor ippd_begin_step would stage for this
+ * step (*bytes) and the capacity of a staging slot of this layout (*capacity, a bound over
+ * every admissible step).  Same argument checks as ippd_begin_step; needs no bound cache. */
+int ippd_step_descriptor_bytes(const ippd_layout_t* layout, const int32_t* active_q,
+                               const int32_t* answer_idx, int32_t n_active, size_t* bytes,
+                               size_t* capacity);
+
 /*
  * ippd_append_kv -- rotate raw keys to their virtual positions (RoPE, fp32 math on an
  * fp64-built table, result rounded to bf16) and store K and V into the cache
- * (paper Sec. 4.2: each new token is appended "with the correct virtual position id").
+ * (paper Sec. 4.2, last paragraph: the token appended at each step carries its virtual position).
  *   kind CONTEXT : ids[n_ids] = prompt ids (host); tokens = all context tokens of those
  *                  prompts, in id order; token i of prompt b gets position i.
  *   kind QUESTION: ids[n_ids] = global question ids (host); tokens = their question
@@ -238,7 +249,9 @@ int ippd_export_mask(ippd_layout_t* layout, int32_t prompt, const int32_t* n_ans
 
 /* Waits for the stream last used with this layout and returns the device error word
  * (0 = none; bit 0 = a bounded wait ran out: IPPD_ERR_TIMEOUT; bit 1 = an id or slot was out of
- * range: IPPD_ERR_INVALID_ARG).  The word is cleared once reported; the outputs of the launches
+ * range: IPPD_ERR_INVALID_ARG; bit 2 = ippd_append_kv was handed a NaN or an infinity:
+ * IPPD_ERR_INVALID_ARG -- the value was stored, and because a key/value row shares its 128-row
+ * tile with other questions' rows, outputs of OTHER questions may be non-finite too).  The word is cleared once reported; the outputs of the launches
  * since the previous poll are then undefined, the cache and the layout stay usable. */
 int ippd_poll_status(ippd_layout_t* layout, int32_t* device_error_word);
 

@@ -12,7 +12,7 @@ from typing import Optional, Sequence
 
 import numpy as np
 
-_LIB_PATH = os.environ.get("IPPD_LIB") or os.path.join(os.path.dirname(os.path.abspath(__file__)), "libippd.so")
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libippd.so")
 if not os.path.exists(_LIB_PATH):
     raise ImportError(f"{_LIB_PATH} is missing: build it with `python -m paper_2609_05707_b200.build`")
 lib = C.CDLL(_LIB_PATH)
@@ -25,7 +25,7 @@ APPEND_CONTEXT, APPEND_QUESTION, APPEND_STEP = 0, 1, 2
 OPT_KERNEL, OPT_LAYERS_PER_CALL, OPT_TILES_PER_SPLIT, OPT_WAIT_LIMIT_US, OPT_PROFILE = 1, 2, 3, 4, 5
 
 EXPORTS = ["ippd_build_layout", "ippd_layout_tables", "ippd_cache_bytes", "ippd_bind_cache", "ippd_set_option",
-           "ippd_begin_step", "ippd_append_kv", "ippd_workspace_bytes", "ippd_decode_attention", "ippd_decode_attention_static",
+           "ippd_begin_step", "ippd_step_descriptor_bytes", "ippd_append_kv", "ippd_workspace_bytes", "ippd_decode_attention", "ippd_decode_attention_static",
            "ippd_decode_step_host", "ippd_decode_step_host_async", "ippd_host_steps_wait", "ippd_step_stage_bytes", "ippd_export_mask", "ippd_poll_status", "ippd_profile_read",
            "ippd_launch_count", "ippd_last_error", "ippd_destroy_layout"]
 
@@ -54,6 +54,7 @@ lib.ippd_cache_bytes.argtypes = [_vp, C.POINTER(_sz), C.POINTER(_sz)]
 lib.ippd_bind_cache.argtypes = [_vp, _vp, _sz, _vp]
 lib.ippd_set_option.argtypes = [_vp, _i32, _i64]
 lib.ippd_begin_step.argtypes = [_vp, _pi32, _pi32, _i32, _vp]
+lib.ippd_step_descriptor_bytes.argtypes = [_vp, _pi32, _pi32, _i32, C.POINTER(_sz), C.POINTER(_sz)]
 lib.ippd_append_kv.argtypes = [_vp, _i32, _i32, _i32, _pi32, _i32, _vp, _vp, _vp]
 lib.ippd_workspace_bytes.argtypes = [_vp, _i32, C.POINTER(_sz)]
 lib.ippd_decode_attention.argtypes = [_vp, _i32, _i32, _vp, _vp, _vp, _sz, _vp]
@@ -155,6 +156,14 @@ class Layout:
     def begin_step(self, active_q, answer_idx, stream: int = 0):
         a, s = _i32arr(active_q), _i32arr(answer_idx)
         _check(lib.ippd_begin_step(self._h, _p(a), _p(s), len(a), stream), "ippd_begin_step")
+
+    def step_descriptor_bytes(self, active_q, answer_idx):
+        """(bytes of the descriptor begin_step would stage for this step, capacity of a staging slot); host-only."""
+        a, s = _i32arr(active_q), _i32arr(answer_idx)
+        b, c = _sz(), _sz()
+        _check(lib.ippd_step_descriptor_bytes(self._h, _p(a), _p(s), len(a), C.byref(b), C.byref(c)),
+               "ippd_step_descriptor_bytes")
+        return b.value, c.value
 
     def append_kv(self, layer_begin: int, layer_count: int, kind: int, ids, k_raw, v_raw, stream: int = 0):
         i = _i32arr(ids if ids is not None else [])

@@ -19,8 +19,6 @@ def _newest_source_mtime() -> float:
 
 def build(force: bool = False, verbose: bool = False) -> str:
     """Builds libippd.so if it is missing or older than its sources; returns its path."""
-    if os.environ.get("IPPD_LIB"):  # an explicitly chosen library (A/B comparisons): nothing to build
-        return os.environ["IPPD_LIB"]
     if not force and os.path.exists(LIB) and os.path.getmtime(LIB) >= _newest_source_mtime():
         return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
@@ -28,7 +26,6 @@ def build(force: bool = False, verbose: bool = False) -> str:
            "-shared", "-Xcompiler", "-fPIC", "-cudart", "static", "-o", LIB]
     if verbose:
         cmd += ["-Xptxas", "-v"]
-    cmd += os.environ.get("IPPD_NVCC_FLAGS", "").split()  # e.g. -DIPPD_TC_TIMING for the diagnostic build
     cmd += [os.path.join(CSRC, s) for s in SOURCES]
     res = subprocess.run(cmd, capture_output=True, text=True)
     if verbose or res.returncode != 0:

@@ -3,6 +3,7 @@
 
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <new>
 
 #include "ippd_attn_mma.cuh"
@@ -66,6 +67,53 @@ struct ippd_layout {
   cudaEvent_t hs_ev_in[2] = {}, hs_ev_done[2] = {}, hs_ev_out[2] = {};
   int64_t hs_count = 0;
 };
+
+static size_t ceil_div_sz(size_t a, size_t b) { return (a + b - 1) / b; }
+
+static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// Offsets of the parts of a step descriptor (each 16-byte aligned) and its total size.
+struct StepBlobLayout {
+  size_t off_q, off_s, off_rb, off_u, off_tb, off_tt, off_tp, off_pos, total;
+};
+static StepBlobLayout step_blob_layout(size_t A, size_t n_rb, size_t n_units, size_t n_tiles, size_t n_pieces) {
+  StepBlobLayout b;
+  b.off_q = 0;
+  b.off_s = align_up(b.off_q + A * 4, 16);
+  b.off_rb = align_up(b.off_s + A * 4, 16);
+  b.off_u = align_up(b.off_rb + n_rb * sizeof(IppdRowBlock), 16);
+  b.off_tb = align_up(b.off_u + n_units * sizeof(IppdUnit), 16);
+  b.off_tt = align_up(b.off_tb + (n_rb + 1) * 4, 16);
+  b.off_tp = align_up(b.off_tt + n_tiles * sizeof(IppdTcTile), 16);
+  b.off_pos = align_up(b.off_tp + n_pieces * sizeof(IppdTcPiece), 16);
+  b.total = align_up(b.off_pos + A * 4, 16) + 16;
+  return b;
+}
+
+// Capacity of a descriptor staging slot: a bound of the descriptor size over every step the layout admits (every
+// question active, every branch full), and of the id list of a CONTEXT / QUESTION append.
+//   row blocks  <= nrb; unit list (mma.sync path) <= max over the split settings of its unit count;
+//   key tiles   <= every row block's context tiles + packed branch tiles; 16 groups of 8 tokens per packed tile and
+//                  at most 16 groups per cache tile of a branch give packed tiles <= branch cache tiles + nrb;
+//   pieces      <= one per (question, cache tile) run + one more wherever a packed tile's per-quarter allotment ends
+//                  inside a run: runs + 4 * packed tiles <= 5 * branch cache tiles + 4 * nrb.
+static size_t ring_capacity(const IppdHostLayout& h) {
+  const size_t nrb = (size_t)ippd_host_max_rowblocks(h);
+  const size_t branch_tiles = (size_t)(h.n_tiles - h.n_ctx_tiles);
+  const int qpr_tc = std::max(1, std::min(IPPD_MAX_ROWS_PER_BLOCK / h.G, 64));
+  const int qpr_mma = std::max(1, 64 / h.G);
+  size_t ctx_tiles_all_blocks = 0;  // whichever kernel path is selected later
+  for (int b = 0; b < h.B; ++b) {
+    const size_t blocks = (size_t)(h.q_count[b] + std::min(qpr_tc, qpr_mma) - 1) / std::min(qpr_tc, qpr_mma);
+    ctx_tiles_all_blocks += (size_t)(h.ctx_tile_off[b + 1] - h.ctx_tile_off[b]) * blocks;
+  }
+  const size_t nrb_any = std::max(nrb, (size_t)ceil_div_sz(h.NQ, 1));  // row blocks never outnumber questions
+  const size_t units = ctx_tiles_all_blocks + branch_tiles + nrb_any + 2048;  // one unit per tile at worst
+  const StepBlobLayout b = step_blob_layout((size_t)h.NQ, nrb_any, units, ctx_tiles_all_blocks + branch_tiles + nrb_any,
+                                            5 * branch_tiles + 4 * nrb_any);
+  const size_t ids = ((size_t)2 * std::max(h.NQ, h.B) + 4) * 4;
+  return align_up(std::max(b.total, ids) + 256, 256);  // the upload kernel moves 16-byte words
+}
 
 // Launch with the programmatic-serialisation attribute: the kernel may be scheduled while its predecessor in the
 // stream still runs and calls pdl_wait() before it touches global memory.
@@ -242,20 +290,8 @@ extern "C" int ippd_bind_cache(ippd_layout_t* L, void* dev_cache, size_t bytes, 
                                                                                 h.geom.head_dim, h.geom.rope_theta);
   CUDA_TRY(cudaGetLastError());
   L->launches++;
-  // descriptor ring: the largest blob is a step plan (active list, row blocks, units or tiles + pieces) or an
-  // append id list
-  size_t nrb = (size_t)ippd_host_max_rowblocks(h);
-  size_t branch_tiles = (size_t)(h.n_tiles - h.n_ctx_tiles);
-  size_t ctx_tiles_all_blocks = 0;
-  for (int b = 0; b < h.B; ++b)
-    ctx_tiles_all_blocks += (size_t)(h.ctx_tile_off[b + 1] - h.ctx_tile_off[b]) * (size_t)((h.q_count[b] + 0) / 1 + 1);
-  ctx_tiles_all_blocks = std::min(ctx_tiles_all_blocks, (size_t)h.n_ctx_tiles * std::max<size_t>(1, nrb));
-  size_t cap = 4096 + (size_t)h.NQ * 8 + nrb * sizeof(IppdRowBlock) + (nrb + 1) * 4 +
-               ((size_t)h.n_tiles + ctx_tiles_all_blocks + nrb + 2048) * sizeof(IppdUnit) +
-               (ctx_tiles_all_blocks + branch_tiles + 4 * nrb) * sizeof(IppdTcTile) +
-               (2 * branch_tiles + 4 * nrb + 16) * sizeof(IppdTcPiece) + (size_t)(h.NQ + h.B + 2) * 8;
-  cap = (std::min<size_t>(cap, (size_t)256 << 20) + 255) & ~(size_t)255;  // the upload kernel moves 16-byte words
-  L->ring_cap = cap;
+  L->ring_cap = ring_capacity(h);
+  const size_t cap = L->ring_cap;
   for (int i = 0; i < kRingSlots; ++i) {
     CUDA_TRY(cudaHostAlloc((void**)&L->ring_host[i], cap, cudaHostAllocMapped));
     CUDA_TRY(cudaHostGetDevicePointer((void**)&L->ring_host_dev[i], L->ring_host[i], 0));
@@ -318,8 +354,6 @@ static int ring_upload(ippd_layout* L, const void* blob, size_t bytes, cudaStrea
   return ring_flush(L, stream);
 }
 
-static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
-
 extern "C" int ippd_begin_step(ippd_layout_t* L, const int32_t* active_q, const int32_t* answer_idx,
                                int32_t A, void* stream_) {
   if (!L) { ippd_set_error("ippd_begin_step: NULL layout"); return IPPD_ERR_INVALID_ARG; }
@@ -330,16 +364,10 @@ extern "C" int ippd_begin_step(ippd_layout_t* L, const int32_t* active_q, const 
   int rc = ippd_host_plan_step(L->h, active_q, answer_idx, A, plan_layers(L), &L->plan);
   if (rc != IPPD_OK) return rc;
   const IppdStepPlan& P = L->plan;
-  // blob: [act_q | act_s | row blocks | units], each 16-byte aligned
-  size_t off_q = 0;
-  size_t off_s = align_up(off_q + (size_t)A * 4, 16);
-  size_t off_rb = align_up(off_s + (size_t)A * 4, 16);
-  size_t off_u = align_up(off_rb + P.rbs.size() * sizeof(IppdRowBlock), 16);
-  size_t off_tb = align_up(off_u + P.units.size() * sizeof(IppdUnit), 16);
-  size_t off_tt = align_up(off_tb + P.rb_tile_begin.size() * 4, 16);
-  size_t off_tp = align_up(off_tt + P.tc_tiles.size() * sizeof(IppdTcTile), 16);
-  size_t off_pos = align_up(off_tp + P.tc_pieces.size() * sizeof(IppdTcPiece), 16);
-  size_t total = align_up(off_pos + (size_t)A * 4, 16) + 16;
+  // blob: [act_q | act_s | row blocks | units | tile prefix | tiles | pieces | positions], each 16-byte aligned
+  const StepBlobLayout bl = step_blob_layout((size_t)A, P.rbs.size(), P.units.size(), P.tc_tiles.size(), P.tc_pieces.size());
+  const size_t off_q = bl.off_q, off_s = bl.off_s, off_rb = bl.off_rb, off_u = bl.off_u, off_tb = bl.off_tb,
+               off_tt = bl.off_tt, off_tp = bl.off_tp, off_pos = bl.off_pos, total = bl.total;
   std::vector<char> blob(total, 0);
   if (A) {
     memcpy(blob.data() + off_q, P.act_q.data(), (size_t)A * 4);
@@ -377,6 +405,17 @@ extern "C" int ippd_begin_step(ippd_layout_t* L, const int32_t* active_q, const 
   for (const IppdRowBlock& rb : P.rbs) L->step_needs_merge |= rb.n_seg > 1;
   L->have_step = true;
   L->last_stream = stream;
+  return IPPD_OK;
+}
+
+extern "C" int ippd_step_descriptor_bytes(const ippd_layout_t* L, const int32_t* active_q, const int32_t* answer_idx,
+                                          int32_t A, size_t* bytes, size_t* capacity) {
+  if (!L || !bytes || !capacity) { ippd_set_error("ippd_step_descriptor_bytes: NULL argument"); return IPPD_ERR_INVALID_ARG; }
+  IppdStepPlan plan;
+  int rc = ippd_host_plan_step(L->h, active_q, answer_idx, A, plan_layers(L), &plan);
+  if (rc != IPPD_OK) return rc;
+  *bytes = step_blob_layout((size_t)A, plan.rbs.size(), plan.units.size(), plan.tc_tiles.size(), plan.tc_pieces.size()).total;
+  *capacity = ring_capacity(L->h);
   return IPPD_OK;
 }
 
@@ -518,14 +557,19 @@ static size_t scratch_need(const ippd_layout* L, int layer_count, size_t* o_byte
 template <int D>
 static int launch_attention(ippd_layout* L, const IppdDev& d, int layer_begin, int layer_count, const void* q_raw,
                             void* out, float* part_o, float* part_ml, cudaStream_t stream, bool marks) {
-  static bool attr_set[64] = {};
-  int dev = L->device >= 0 && L->device < 64 ? L->device : 0;
-  if (!attr_set[dev]) {
-    CUDA_TRY(cudaFuncSetAttribute(ippd_attn_mma_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                  MmaCfg<D>::SMEM));
-    CUDA_TRY(cudaFuncSetAttribute(ippd_attn_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                  tc_smem_bytes<D>()));
-    attr_set[dev] = true;
+  {
+    // once per device and head size; host threads making their first calls at the same time take turns
+    static std::mutex mu;
+    static bool attr_set[64] = {};
+    std::lock_guard<std::mutex> lock(mu);
+    int dev = L->device >= 0 && L->device < 64 ? L->device : 0;
+    if (!attr_set[dev]) {
+      CUDA_TRY(cudaFuncSetAttribute(ippd_attn_mma_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    MmaCfg<D>::SMEM));
+      CUDA_TRY(cudaFuncSetAttribute(ippd_attn_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    tc_smem_bytes<D>()));
+      attr_set[dev] = true;
+    }
   }
   const IppdStepDev& S = L->step_dev;
   const int Hkv = L->h.geom.n_kv_heads;
@@ -620,6 +664,7 @@ extern "C" int ippd_decode_attention(ippd_layout_t* L, int32_t layer_begin, int3
 // address a kernel may use comes from cudaGetSymbolAddress, looked up once per device below.
 static __device__ __align__(256) unsigned char g_ippd_static_scratch[IPPD_STATIC_SCRATCH_BYTES];
 static void* g_static_scratch_addr[64] = {};
+static std::mutex g_static_scratch_mu;  // guards the table above: first calls may come from several host threads
 
 extern "C" int ippd_decode_attention_static(ippd_layout_t* L, int32_t layer_begin, int32_t layer_count,
                                             const void* q_raw, void* out, void* stream_) {
@@ -654,15 +699,20 @@ extern "C" int ippd_decode_attention_static(ippd_layout_t* L, int32_t layer_begi
                      "; pass fewer layers per call or raise IPPD_OPT_TILES_PER_SPLIT");
       return IPPD_ERR_CAPACITY;
     }
-    if (!g_static_scratch_addr[dev]) {
-      // first call on this device (it is the current one): resolve the symbol to its device address
-      void* p = nullptr;
-      CUDA_TRY(cudaGetSymbolAddress(&p, g_ippd_static_scratch));
-      if (!p) { ippd_set_error("ippd_decode_attention_static: scratch symbol has no device address"); return IPPD_ERR_CUDA; }
-      g_static_scratch_addr[dev] = p;
+    void* base = nullptr;
+    {
+      std::lock_guard<std::mutex> lock(g_static_scratch_mu);
+      if (!g_static_scratch_addr[dev]) {
+        // first call on this device (it is the current one): resolve the symbol to its device address
+        void* p = nullptr;
+        CUDA_TRY(cudaGetSymbolAddress(&p, g_ippd_static_scratch));
+        if (!p) { ippd_set_error("ippd_decode_attention_static: scratch symbol has no device address"); return IPPD_ERR_CUDA; }
+        g_static_scratch_addr[dev] = p;
+      }
+      base = g_static_scratch_addr[dev];
     }
-    part_o = (float*)g_static_scratch_addr[dev];
-    part_ml = (float*)((char*)g_static_scratch_addr[dev] + o_bytes);
+    part_o = (float*)base;
+    part_ml = (float*)((char*)base + o_bytes);
   }
   {
     int rc = ring_flush(L, stream);  // the step's descriptor, unless a STEP append carried it along
@@ -844,6 +894,7 @@ extern "C" int ippd_poll_status(ippd_layout_t* L, int32_t* word) {
   if (*word) CUDA_TRY(cudaMemset(L->d_error, 0, sizeof(int32_t)));  // reported once; the layout stays usable
   if (*word & IPPD_ERRBIT_TIMEOUT) { ippd_set_error("a bounded device-side wait ran out"); return IPPD_ERR_TIMEOUT; }
   if (*word & IPPD_ERRBIT_RANGE) { ippd_set_error("an id or slot was out of range on the device"); return IPPD_ERR_INVALID_ARG; }
+  if (*word & IPPD_ERRBIT_NONFINITE) { ippd_set_error("ippd_append_kv was handed a NaN or an infinity"); return IPPD_ERR_INVALID_ARG; }
   return IPPD_OK;
 }
 
@@ -868,16 +919,6 @@ extern "C" int ippd_profile_read(ippd_layout_t* L, double* attention_ms, double*
   if (n_attention) *n_attention = n_att;
   return IPPD_OK;
 }
-
-#ifdef IPPD_TC_TIMING
-extern "C" int ippd_debug_read_timing(unsigned long long* out16) {
-  CUDA_TRY(cudaDeviceSynchronize());
-  CUDA_TRY(cudaMemcpyFromSymbol(out16, g_tc_timing, sizeof(unsigned long long) * 16));
-  unsigned long long z[16] = {};
-  CUDA_TRY(cudaMemcpyToSymbol(g_tc_timing, z, sizeof(z)));
-  return IPPD_OK;
-}
-#endif
 
 extern "C" int64_t ippd_launch_count(const ippd_layout_t* L) { return L ? L->launches : 0; }
 

@@ -184,29 +184,9 @@ constexpr int tc_smem_bytes() {
   return IPPD_TC_NBUF * 16 * (D / 8) * 128 + (int)sizeof(TcShared);
 }
 
-#ifdef IPPD_TC_TIMING
-// Diagnostic build only (-DIPPD_TC_TIMING): cycles per activity, summed over all CTAs, taken on lane 0 of the producer
-// warp (0), the P V issuer (1), the S issuer (18) and one softmax warp (4: warpgroup 0, rows 0..31).  Slots:
-//   0 producer waits for a free ring buffer   1 S issuer waits for Q~   2 ... for a K tile   3 ... for the P V product
-//   that frees the S buffer   4 P V issuer waits for a V tile   5 ... for P   6 ... for the epilogue to free O
-//   7 softmax waits for S   8 TMEM load + masked maximum   9 Q~ staging   10 epilogue   11 quarter barrier
-//   12 whole kernel (thread 0)   13 exp2 + P store   14 wait for the store + arrive   15 softmax waits for a P V product
-__device__ unsigned long long g_tc_timing[16];
-#define TC_T0() long long _t0 = clock64()
-#define TC_TREC(slot, t0) do { if ((threadIdx.x & 31) == 0 && (threadIdx.x < 64 || (threadIdx.x >> 5) == 4 || (threadIdx.x >> 5) == 18)) atomicAdd(&g_tc_timing[slot], (unsigned long long)(clock64() - (t0))); } while (0)
-#define TC_T1(slot) TC_TREC(slot, _t0)
-#define TC_MARK(var) long long var = clock64()
-#define TC_REMARK(var) var = clock64()
-#else
-#define TC_T0()
-#define TC_T1(slot)
-#define TC_TREC(slot, t0)
-#define TC_MARK(var)
-#define TC_REMARK(var)
-#endif
 
 // Bounded wait that also gives up when another role has raised the abort flag.
-__device__ __forceinline__ bool tc_wait_impl(uint64_t* bar, uint32_t parity, const IppdDev& L, TcShared* sh) {
+__device__ __forceinline__ bool tc_wait(uint64_t* bar, uint32_t parity, const IppdDev& L, TcShared* sh) {
   if (mbar_try_wait(bar, parity)) return true;
   if (L.wait_limit_ns == 0) {  // "never wait": a phase still incomplete after one (briefly suspending) probe fails
     sh->abort_flag = 1;
@@ -227,13 +207,6 @@ __device__ __forceinline__ bool tc_wait_impl(uint64_t* bar, uint32_t parity, con
   }
   return true;
 }
-// `slot` only labels the wait in the diagnostic timing build.
-__device__ __forceinline__ bool tc_wait(uint64_t* bar, uint32_t parity, const IppdDev& L, TcShared* sh, int slot = 15) {
-  TC_T0();
-  bool r = tc_wait_impl(bar, parity, L, sh);
-  TC_T1(slot);
-  return r;
-}
 
 #include "ippd_attn_tc_softmax.cuh"
 
@@ -251,9 +224,6 @@ ippd_attn_tc_kernel(IppdDev L, IppdStepDev S, IppdTcArgs A, const __nv_bfloat16*
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int Hkv = L.Hkv;
   pdl_trigger();  // the merge kernel may be scheduled as soon as SMs become free
-#ifdef IPPD_TC_TIMING
-  const long long t_kernel0 = clock64();
-#endif
   const long long g0 = (long long)blockIdx.x * A.chunk;
   const long long g1 = min(A.total_tiles, g0 + A.chunk);
 
@@ -309,7 +279,7 @@ ippd_attn_tc_kernel(IppdDev L, IppdStepDev S, IppdTcArgs A, const __nv_bfloat16*
         const int groups = (ti.rows + 7) >> 3;
         for (int kv = 0; kv < 2 && ok; ++kv, ++n) {
           uint32_t buf = n % IPPD_TC_NBUF, ph = (n / IPPD_TC_NBUF) & 1;
-          if (lane == 0) ok = tc_wait(&sh->kv_empty[buf], ph ^ 1, L, sh, 0);
+          if (lane == 0) ok = tc_wait(&sh->kv_empty[buf], ph ^ 1, L, sh);
           ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
           if (!ok) break;
           uint8_t* dst = ring + buf * TILE_BYTES;
@@ -358,11 +328,11 @@ ippd_attn_tc_kernel(IppdDev L, IppdStepDev S, IppdTcArgs A, const __nv_bfloat16*
         const int nt = sg.t_end - sg.t_begin;
         for (int i = 0; i < nt; ++i, ++jt) {
           const uint32_t nb = 2 * jt + 1, buf = nb % IPPD_TC_NBUF, ph = (nb / IPPD_TC_NBUF) & 1;
-          if (!tc_wait(&sh->kv_full[buf], ph, L, sh, 4)) { ok = false; break; }
-          if (!tc_wait(&sh->p_full[jt & 1], (jt >> 1) & 1, L, sh, 5)) { ok = false; break; }
+          if (!tc_wait(&sh->kv_full[buf], ph, L, sh)) { ok = false; break; }
+          if (!tc_wait(&sh->p_full[jt & 1], (jt >> 1) & 1, L, sh)) { ok = false; break; }
           if (i == 0 && nseg > 0) {
             // the epilogue of the previous segment has read O
-            if (!tc_wait(&sh->o_free, (nseg - 1) & 1, L, sh, 6)) { ok = false; break; }
+            if (!tc_wait(&sh->o_free, (nseg - 1) & 1, L, sh)) { ok = false; break; }
           }
           tc_fence_after();
           const uint32_t v_lo = ring_lo_v + buf * (TILE_BYTES >> 4);
@@ -402,12 +372,12 @@ ippd_attn_tc_kernel(IppdDev L, IppdStepDev S, IppdTcArgs A, const __nv_bfloat16*
           atomicOr(L.error_word, IPPD_ERRBIT_TIMEOUT);
           break;
         }
-        if (!tc_wait(&sh->q_full, nseg & 1, L, sh, 1)) break;
+        if (!tc_wait(&sh->q_full, nseg & 1, L, sh)) break;
         const uint32_t a_tmem = tQ + (nseg & 1) * 64;
         for (int i = 0; i < nt; ++i, ++jt) {
           const uint32_t nb = 2 * jt, buf = nb % IPPD_TC_NBUF, ph = (nb / IPPD_TC_NBUF) & 1;
-          if (!tc_wait(&sh->kv_full[buf], ph, L, sh, 2)) { ok = false; break; }
-          if (jt >= 2 && !tc_wait(&sh->pv_done[jt & 1], ((jt - 2) >> 1) & 1, L, sh, 3)) { ok = false; break; }
+          if (!tc_wait(&sh->kv_full[buf], ph, L, sh)) { ok = false; break; }
+          if (jt >= 2 && !tc_wait(&sh->pv_done[jt & 1], ((jt - 2) >> 1) & 1, L, sh)) { ok = false; break; }
           tc_fence_after();
           const int rows_i = sh->meta[jt % IPPD_TC_NMETA].rows;  // published by the K buffer's barrier
           const uint32_t idesc = tc_idesc(128, (rows_i + 15) & ~15, 0);
@@ -428,9 +398,6 @@ ippd_attn_tc_kernel(IppdDev L, IppdStepDev S, IppdTcArgs A, const __nv_bfloat16*
     tc_softmax_role<D>(L, S, A, sh, tmem, g0, g1, q_raw, out, part_o, part_ml);
   }
 
-#ifdef IPPD_TC_TIMING
-  if (tid == 0) atomicAdd(&g_tc_timing[12], (unsigned long long)(clock64() - t_kernel0));
-#endif
   // ---- teardown: every role gets here (all waits are bounded) ----
   tc_fence_before();
   __syncthreads();

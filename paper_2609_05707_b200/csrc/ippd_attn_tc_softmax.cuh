@@ -46,9 +46,7 @@ __device__ __forceinline__ unsigned short tc_bf16_ceil_bits(float x) {
 // the abort flag) still makes the passes it owes (see the end of tc_softmax_role), so nobody is left waiting.
 // All lanes of a warp execute every wait converged on one barrier and so see the same outcome.
 __device__ __forceinline__ void tc_quad_sync(int warp) {
-  TC_T0();
   asm volatile("bar.sync %0, 128;" ::"r"(2 + (warp & 3)) : "memory");
-  TC_T1(11);
 }
 // A softmax warp that gives up makes the passes it still owes: `owed_here` in its current segment, plus one per tile
 // and three per epilogue for every later segment of the CTA's slice [g, g1) (g = first tile after the current segment;
@@ -88,7 +86,6 @@ __device__ __forceinline__ void tc_softmax_role(const IppdDev& L, const IppdStep
   // column c holds the bf16 pair (2c, 2c+1) of the row) and signals the MMA warp.  The buffer was last read by the S
   // MMAs of the segment before the previous one, which are long complete.
   auto stage_q = [&](const TcSegment& sq, uint32_t qbuf) {
-    TC_MARK(t_stage);
     const IppdRowBlock rb = S.rbs[sq.rb];
     const int nrows = rb.n_act * G;
     uint32_t wlo[NW], whi[NW];  // rotated pairs d in [2*NW*wg, 2*NW*(wg+1)) and the same + D/2
@@ -129,7 +126,6 @@ __device__ __forceinline__ void tc_softmax_role(const IppdDev& L, const IppdStep
     tc_fence_before();
     __syncwarp();
     if (lane == 0) mbar_arrive(&sh->q_full);
-    TC_TREC(9, t_stage);
   };
 
   int gofs = 0;  // position in the CTA's slice, relative to g0 (a 32-bit value: this role is short of registers)
@@ -154,9 +150,8 @@ __device__ __forceinline__ void tc_softmax_role(const IppdDev& L, const IppdStep
     float m_ref = -INFINITY, l_sum = 0.f;  // l_sum: this thread's part of the row sum
     const int nt = sg.t_end - sg.t_begin;
     for (int i = 0; i < nt; ++i, ++jt) {
-      if (!tc_wait(&sh->s_full[jt & 1], (jt >> 1) & 1, L, sh, 7)) { tc_quad_give_up(A.rb_tile_begin, S.n_rb, A.T1, g0 + gofs, g1, nt - i + 3, warp); return; }
+      if (!tc_wait(&sh->s_full[jt & 1], (jt >> 1) & 1, L, sh)) { tc_quad_give_up(A.rb_tile_begin, S.n_rb, A.T1, g0 + gofs, g1, nt - i + 3, warp); return; }
       tc_fence_after();
-      TC_MARK(t_phase);
       // the tile's description was staged by the producer before its K copy, which S(jt) has consumed
       const TcMeta& meta = sh->meta[jt % IPPD_TC_NMETA];
       const int tile_rows = meta.rows, n_pieces = meta.n_pieces;
@@ -241,9 +236,7 @@ __device__ __forceinline__ void tc_softmax_role(const IppdDev& L, const IppdStep
       // barrier also orders every owner's S loads before the P stores below, which overwrite S columns of other owners
       const unsigned short mbits = tc_bf16_ceil_bits(mloc);
       sh->xmax[jt & 1][wg][row] = mbits;
-      TC_TREC(8, t_phase);
       tc_quad_sync(warp);
-      TC_REMARK(t_phase);
       float mt;
       {
         const unsigned short b0 = sh->xmax[jt & 1][0][row], b1 = sh->xmax[jt & 1][1][row];
@@ -261,7 +254,7 @@ __device__ __forceinline__ void tc_softmax_role(const IppdDev& L, const IppdStep
       }
       if (i > 0 && __any_sync(FULL, grow)) {
         // rare: rescale my quarter of the O row, which needs PV(jt-1) to have finished
-        if (!tc_wait(&sh->pv_done[(jt - 1) & 1], ((jt - 1) >> 1) & 1, L, sh, 15)) { tc_quad_give_up(A.rb_tile_begin, S.n_rb, A.T1, g0 + gofs, g1, nt - i - 1 + 3, warp); return; }
+        if (!tc_wait(&sh->pv_done[(jt - 1) & 1], ((jt - 1) >> 1) & 1, L, sh)) { tc_quad_give_up(A.rb_tile_begin, S.n_rb, A.T1, g0 + gofs, g1, nt - i - 1 + 3, warp); return; }
         tc_fence_after();
         uint32_t o[DQ];
         if constexpr (DQ == 32) { TC_LD32(tO + lane_base + wg * DQ, o); } else { TC_LD16(tO + lane_base + wg * DQ, o); }
@@ -288,13 +281,10 @@ __device__ __forceinline__ void tc_softmax_role(const IppdDev& L, const IppdStep
         }
         TC_ST16(tP, p);
       }
-      TC_TREC(13, t_phase);
-      TC_REMARK(t_phase);
       tc_wait_st();  // the P words and a possible O rescale
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&sh->p_full[jt & 1]);
-      TC_TREC(14, t_phase);
     }
     // ---- the next segment's Q~ goes to the other TMEM buffer now, so that the MMA warp can start its first S tiles
     // while this segment's epilogue runs ----
@@ -304,7 +294,6 @@ __device__ __forceinline__ void tc_softmax_role(const IppdDev& L, const IppdStep
     if (have_next) stage_q(nx, (nseg + 1) & 1);
     // ---- epilogue: total row sum (exchanged through my row's own maxima slots: low half in parity 0, high half in
     // parity 1), wait for the last PV, store my quarter of the O row ----
-    TC_MARK(t_epi);
     tc_quad_sync(warp);  // my row's other owners have read the last tile's maxima
     {
       const uint32_t lb = __float_as_uint(l_sum);
@@ -317,7 +306,7 @@ __device__ __forceinline__ void tc_softmax_role(const IppdDev& L, const IppdStep
     for (int w = 0; w < IPPD_TC_NWG; ++w)
       l_tot += __uint_as_float((uint32_t)sh->xmax[0][w][row] | ((uint32_t)sh->xmax[1][w][row] << 16));
     tc_quad_sync(warp);  // the slots go back to the maxima of the next tiles
-    if (!tc_wait(&sh->pv_done[(jt - 1) & 1], ((jt - 1) >> 1) & 1, L, sh, 15)) { tc_quad_give_up(A.rb_tile_begin, S.n_rb, A.T1, g0 + gofs, g1, 0, warp); return; }
+    if (!tc_wait(&sh->pv_done[(jt - 1) & 1], ((jt - 1) >> 1) & 1, L, sh)) { tc_quad_give_up(A.rb_tile_begin, S.n_rb, A.T1, g0 + gofs, g1, 0, warp); return; }
     tc_fence_after();
     {
       const bool valid_row = row < nrows;
@@ -366,7 +355,6 @@ __device__ __forceinline__ void tc_softmax_role(const IppdDev& L, const IppdStep
     tc_fence_before();
     __syncwarp();
     if (lane == 0) mbar_arrive(&sh->o_free);
-    TC_TREC(10, t_epi);
     ++nseg;
     sg = nx;
     gofs = (int)(g_next - g0);

@@ -93,6 +93,19 @@ ippd_append_kernel(IppdDev L, IppdStepDev S, IppdAppendArgs a, int layer_begin,
   uint4 khi = *reinterpret_cast<const uint4*>(k_raw + src + D / 2);
   uint4 vlo = *reinterpret_cast<const uint4*>(v_raw + src);
   uint4 vhi = *reinterpret_cast<const uint4*>(v_raw + src + D / 2);
+  {
+    // A NaN or an infinity (bf16: all exponent bits set) is stored like any value but reported: a cache row shares
+    // its 128-row tile with rows of other questions, and 0 x NaN would reach their outputs too.
+    const uint32_t* w[4] = {reinterpret_cast<const uint32_t*>(&klo), reinterpret_cast<const uint32_t*>(&khi),
+                            reinterpret_cast<const uint32_t*>(&vlo), reinterpret_cast<const uint32_t*>(&vhi)};
+    bool bad = false;
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+      for (int e = 0; e < 4; ++e)
+        bad |= (w[i][e] & 0x7F800000u) == 0x7F800000u || (w[i][e] & 0x00007F80u) == 0x00007F80u;
+    if (bad) atomicOr(L.error_word, IPPD_ERRBIT_NONFINITE);
+  }
   const float2* cs = L.rope + (size_t)pos * (D / 2) + c * 8;
   const __nv_bfloat162* pl = reinterpret_cast<const __nv_bfloat162*>(&klo);
   const __nv_bfloat162* ph = reinterpret_cast<const __nv_bfloat162*>(&khi);

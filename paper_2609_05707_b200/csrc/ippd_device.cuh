@@ -8,6 +8,7 @@
 
 #define IPPD_ERRBIT_TIMEOUT 1
 #define IPPD_ERRBIT_RANGE 2
+#define IPPD_ERRBIT_NONFINITE 4
 
 // Everything a kernel needs to know about the cache and the ragged tables.
 struct IppdDev {

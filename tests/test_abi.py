@@ -81,3 +81,27 @@ def test_host_argument_checks():
     na = np.array([2], dtype=np.int32)
     assert B.lib.ippd_export_mask(lay._h, 0, na.ctypes.data_as(C.POINTER(C.c_int32)), None, C.byref(cnt)) == 0
     assert cnt.value == 16 + 4 + 2
+
+
+@pytest.mark.parametrize("branch_tokens", [300, 4096, 8192])
+def test_step_descriptor_fits_its_staging_slot_for_long_branches(branch_tokens):
+    # The per-quarter packing of the branch tiles may cut a full 16-group run into several pieces; the staging slot is
+    # sized for that.  Plans the last admissible step of layouts whose branches span many cache tiles (host-only).
+    r = np.random.default_rng(branch_tokens)
+    for G, hq in [(4, 8), (1, 2), (8, 16)]:
+        qc = [32, 5, 70]
+        nq = sum(qc)
+        ql = r.integers(1, 60, nq)
+        mn = np.maximum(1, branch_tokens - ql).astype(np.int32)
+        lay = B.Layout(B.make_geometry(2, hq, hq // G, 128, 5e5), [1000, 0, 130], qc, ql, mn)
+        for kernel in (1, 2):
+            lay.set_option(B.OPT_KERNEL, kernel)
+            for tps in (0, 1):
+                lay.set_option(B.OPT_TILES_PER_SPLIT, tps)
+                act = np.arange(nq, dtype=np.int32)
+                for idx in (mn - 1, np.minimum(mn - 1, r.integers(0, branch_tokens, nq))):
+                    need, cap = lay.step_descriptor_bytes(act, idx.astype(np.int32))
+                    assert 0 < need <= cap, (G, kernel, tps, need, cap)
+        # a subset of the questions can only need less
+        need_sub, cap = lay.step_descriptor_bytes(act[::3], (mn - 1)[::3])
+        assert need_sub <= cap
