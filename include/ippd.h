@@ -237,8 +237,10 @@ int ippd_host_steps_wait(ippd_layout_t* layout, void* stream);
 
 /*
  * ippd_export_mask -- test aid: the dense IPPD mask M_fin (paper Sec. 4.1 mask equations)
- * of ONE prompt's stacked sequence as the kernels realise it, written by a device
- * kernel from the device tables.  Sequence order: context tokens, question blocks,
+ * of ONE prompt's stacked sequence, written by a device kernel that evaluates the library's
+ * visibility rule (context of the own prompt; own branch slots up to the own slot) on the
+ * device tables.  It restates that rule; it does not replay the tiles and packed branch
+ * pieces the attention kernels walk.  Sequence order: context tokens, question blocks,
  * then answer tokens step by step (for t = 0.. : every question of the prompt, in
  * order, with n_answer[k] > t).  n_answer[Q_b] (host) gives how many answer tokens each
  * question of the prompt has.  host_out: [n, n] bytes (1 = attend), row-major, n

@@ -36,12 +36,21 @@ class Runner:
             self.layout.set_option(B.OPT_TILES_PER_SPLIT, tiles_per_split)
         self.layers_per_call = layers_per_call or g.n_layers
         nbytes, _ = self.layout.cache_bytes()
-        self.cache = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
+        self.cache = self.alloc_bytes(nbytes, "cache")
         self.stream = torch.cuda.current_stream(self.device).cuda_stream
         self.layout.bind_cache(self.cache, self.stream)
-        self.workspace = torch.empty(self.layout.workspace_bytes(self.layers_per_call), dtype=torch.uint8,
-                                     device=self.device)
+        self.workspace = self.alloc_bytes(self.layout.workspace_bytes(self.layers_per_call), "workspace")
         self.out_torch_dtype = torch.float32 if out_dtype == B.F32 else torch.bfloat16
+
+    def alloc_bytes(self, nbytes: int, what: str) -> torch.Tensor:
+        """Device buffer handed to the library (uint8, 256-byte aligned).  Subclasses may surround it with guard bands."""
+        return torch.empty(nbytes, dtype=torch.uint8, device=self.device)
+
+    def alloc_out(self, n_active: int) -> torch.Tensor:
+        g = self.wl.geom
+        shape = (g.n_layers, n_active, g.n_q_heads, g.head_dim)
+        n = int(np.prod(shape)) * (4 if self.out_torch_dtype == torch.float32 else 2)
+        return self.alloc_bytes(n, "out").view(self.out_torch_dtype).view(shape)
 
     # ------------------------------------------------------------------ prefill stand-in
     def load_header(self, prompts: Optional[Sequence[int]] = None):
@@ -75,7 +84,7 @@ class Runner:
         g = self.wl.geom
         A = len(act)
         if out is None:
-            out = torch.empty((g.n_layers, A, g.n_q_heads, g.head_dim), dtype=self.out_torch_dtype, device=self.device)
+            out = self.alloc_out(A)
         self.layout.begin_step(act, answer_idx, self.stream)
         if A == 0:
             return out

@@ -39,17 +39,48 @@ def gate(got: np.ndarray, want: np.ndarray, what: str = "", rel: bool = True, ab
     return float(d.max()), float(d.mean()), rms
 
 
+GUARD_BYTES = 4096
+GUARD_FILL = 0xA5
+
+
 class PoisonedRunner(Runner):
     """Runner whose cache starts as the largest finite bf16 (0x7F7F = 3.39e38) in every slot and whose workspace
     starts as NaN: a key or value row used outside its mask, or a stale partial, shows up as inf / NaN / a huge
     error.  (The library's contract is that unwritten cache slots are finite, not that they are never multiplied by a
-    zero probability.)"""
+    zero probability.)
+
+    Every buffer handed to the library (cache, workspace, outputs, staging) sits between two guard bands of
+    GUARD_BYTES filled with GUARD_FILL; `check()` asserts that no band was written.  With the memory checker of the
+    tool chain unavailable on the test machines, this is the evidence that the kernels stay inside their buffers."""
 
     def __init__(self, *a, **kw):
+        self._guarded = []
         super().__init__(*a, **kw)
         self.cache.view(torch.int16).fill_(0x7F7F)
         self.workspace.fill_(0xFF)
         torch.cuda.synchronize()
+
+    def alloc_bytes(self, nbytes, what):
+        assert GUARD_BYTES % 256 == 0
+        padded = (nbytes + 255) // 256 * 256
+        raw = torch.full((padded + 2 * GUARD_BYTES,), GUARD_FILL, dtype=torch.uint8, device=self.device)
+        self._guarded.append((what, raw, nbytes))
+        return raw[GUARD_BYTES:GUARD_BYTES + nbytes]
+
+    def guards_intact(self):
+        torch.cuda.synchronize()
+        for what, raw, nbytes in self._guarded:
+            head = raw[:GUARD_BYTES]
+            tail = raw[GUARD_BYTES + nbytes:]
+            # the bytes between the buffer's end and the next 256-byte boundary belong to the tail band too
+            assert bool((head == GUARD_FILL).all()), f"bytes before the {what} buffer were overwritten"
+            assert bool((tail == GUARD_FILL).all()), f"bytes after the {what} buffer were overwritten"
+        # outputs are allocated per step: keep only the long-lived buffers
+        self._guarded = [g for g in self._guarded if g[0] != "out"]
+
+    def check(self):
+        super().check()
+        self.guards_intact()
 
 
 def oracle_step(wl, s, layer, kv_head, cache=None, step_cache=None, qids=None):

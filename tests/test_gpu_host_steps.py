@@ -41,7 +41,7 @@ def test_host_steps_match_the_oracle(pipelined):
     n_steps = wl.n_steps
     amax = max(len(wl.active(s)) for s in range(n_steps))
     slots = 2 if pipelined else 1
-    stage = torch.empty(slots * run.layout.step_stage_bytes(amax) + 256, dtype=torch.uint8, device=run.device)
+    stage = run.alloc_bytes(slots * run.layout.step_stage_bytes(amax) + 256, "stage")
     stage.fill_(0xFF)
     steps = [_host_inputs(run, wl, s) for s in range(n_steps)]
     outs = [torch.full((g.n_layers, len(a), g.n_q_heads, g.head_dim), float("nan")).pin_memory() for a, _ in steps]
@@ -67,7 +67,7 @@ def test_pipelined_steps_equal_blocking_steps_bit_for_bit():
         run = PoisonedRunner(wl, out_dtype=B.F32)
         run.load_header()
         amax = max(len(wl.active(s)) for s in range(wl.n_steps))
-        stage = torch.empty(2 * run.layout.step_stage_bytes(amax), dtype=torch.uint8, device=run.device)
+        stage = run.alloc_bytes(2 * run.layout.step_stage_bytes(amax), "stage")
         outs = []
         for s in range(wl.n_steps):
             act, (hq, hk, hv) = _host_inputs(run, wl, s)

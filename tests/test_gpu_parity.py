@@ -92,10 +92,13 @@ def test_split_count_does_not_change_the_result(kernel):
         outs.append(out.float().cpu().numpy())
     ref = oracle_step(wl, 2, 0, 1, {})
     gate(np.stack([outs[0][0, i, 4:8] for i in range(9)]), np.stack([ref[k] for k in range(9)]), "splits")
-    # P is rounded to bf16 relative to each split's own running maximum, so different partitions differ at the
-    # level of that rounding (about 2^-9 of an output of size ~0.1); a merge error would be 100x larger
+    # P is rounded to bf16 relative to each split's own running maximum, so different partitions differ at the level
+    # of that rounding: a few 2^-9 of the row's size (row RMS about 0.07 here).  Stated relative to the row RMS so that
+    # a wrong merge weight, which moves a row by a sizeable fraction of its RMS, cannot hide under it.
+    row_rms = np.sqrt((outs[0].astype(np.float64) ** 2).mean(axis=-1, keepdims=True))
     for o in outs[1:]:
-        assert np.abs(o - outs[0]).max() < 1e-3
+        err = np.abs(o.astype(np.float64) - outs[0]) / row_rms
+        assert err.max() <= 1.5e-2 and err.mean() <= 2e-3, (err.max(), err.mean())
 
 
 def test_mask_export_equals_predicates():
@@ -108,6 +111,9 @@ def test_mask_export_equals_predicates():
         qls = [int(v) for v in wl.q_len[k0:k0 + wl.q_count[b]]]
         pos, ctx, qtn, tag = orc.stacked_sequence(0, [int(wl.ctx_len[b])], [qls], [n_answer[b]])
         np.testing.assert_array_equal(got, orc.dense_mask(pos, ctx, qtn))
+    # (this export restates the visibility rule from the device tables; the structural mask the attention kernels
+    # realise through their tiles and packed pieces is pinned through the kernels themselves, by the zero-query test,
+    # whose output is the mean of small-integer values over exactly the visible set)
 
 
 def test_rope_table_and_append_layout():
@@ -154,3 +160,23 @@ def test_a_wait_that_runs_out_is_reported_and_the_layout_stays_usable():
     cache = {}
     for s in range(2):
         compare_step(run, s, [0], range(2), cache, "after-timeout")
+
+
+def test_a_non_finite_key_or_value_is_reported():
+    # K/V rows share 128-row tiles across questions, so a NaN could reach other questions' outputs (0 x NaN); the
+    # append reports it through the error word instead of letting it pass silently.  Nothing faults: the kernel stores
+    # the value and returns normally.
+    wl = W.custom_workload("nan", W.Geometry(1, 8, 2, 128, 5e5), 29, [100], [2], [5, 6], [2, 2])
+    for bad in (float("nan"), float("inf")):
+        run = PoisonedRunner(wl, out_dtype=B.F32)
+        run.load_header()
+        assert run.layout.poll_status() == 0
+        act = wl.active(0)
+        q, k, v = run.step_inputs(0, act)
+        v[0, 1, 1, 77] = bad
+        run.layout.begin_step(act, np.zeros(len(act), dtype=np.int32), run.stream)
+        run.layout.append_kv(0, 1, B.APPEND_STEP, None, k, v, run.stream)
+        with pytest.raises(B.IppdError) as e:
+            run.layout.poll_status()
+        assert e.value.code == B.ERR_INVALID_ARG and "NaN" in str(e.value)
+        assert run.layout.poll_status() == 0  # reported once
