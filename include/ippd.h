@@ -203,10 +203,37 @@ int ippd_decode_attention(ippd_layout_t* layout, int32_t layer_begin, int32_t la
                           void* stream);
 
 /*
+ * ippd_decode_step -- ippd_append_kv(STEP) and ippd_decode_attention in ONE launch (paper Sec. 4.2,
+ * last paragraph: the step's tokens are appended with their virtual positions and attended to in
+ * the same step).  k_raw, v_raw: device bf16 [layer_count, A, Hkv, D], pre-RoPE, the step's tokens in
+ * begin_step order; the other arguments as for ippd_decode_attention.  Inside the attention kernel
+ * one warp per CTA rotates the keys and writes K~ and V into their branch slots just ahead of the
+ * CTA's own loads of those slots, so the cache ends up exactly as after ippd_append_kv(STEP) and the
+ * outputs are those of ippd_decode_attention after it.  Re-running the call rewrites the same slots.
+ * (With IPPD_OPT_KERNEL = 1 the call runs the append kernel and the attention kernel one after the
+ * other.)  Errors as for the two calls it replaces.
+ */
+int ippd_decode_step(ippd_layout_t* layout, int32_t layer_begin, int32_t layer_count, const void* q_raw,
+                     const void* k_raw, const void* v_raw, void* out, void* workspace,
+                     size_t workspace_bytes, void* stream);
+
+/*
+ * ippd_decode_step_grouped -- ippd_decode_step for ALL layers of the step, `layers_per_call` layers per
+ * launch, back to back on `stream`: q_raw [n_layers, A, Hq, D], k_raw / v_raw [n_layers, A, Hkv, D], out
+ * [n_layers, A, Hq, D].  layers_per_call = 1 is the launch pattern of a model whose layer l+1 needs layer
+ * l's output (without the model's own work between the launches); = n_layers is one ippd_decode_step.
+ * The workspace must satisfy ippd_workspace_bytes(layers_per_call); set IPPD_OPT_LAYERS_PER_CALL to the
+ * same value before ippd_begin_step.  Errors as ippd_decode_step.
+ */
+int ippd_decode_step_grouped(ippd_layout_t* layout, int32_t layers_per_call, const void* q_raw,
+                             const void* k_raw, const void* v_raw, void* out, void* workspace,
+                             size_t workspace_bytes, void* stream);
+
+/*
  * ippd_decode_step_host -- one whole decode step from HOST buffers: copies q_raw, k_raw,
  * v_raw (host, pinned or pageable; shapes as above with layer_count = n_layers) into the
- * caller's device staging buffers, runs ippd_begin_step + ippd_append_kv(STEP) +
- * ippd_decode_attention over all layers, copies `out` back to the host and waits for
+ * caller's device staging buffers, runs ippd_begin_step + ippd_decode_step over all layers,
+ * copies `out` back to the host and waits for
  * the stream.  dev_stage must hold the three inputs and the output back to back
  * (ippd_step_stage_bytes).  Same errors as the calls it wraps.
  */
@@ -300,6 +327,19 @@ int ippd_profile_read(ippd_layout_t* layout, double* attention_ms, double* merge
 #define IPPD_STATIC_SCRATCH_BYTES (64u << 20)
 int ippd_decode_attention_static(ippd_layout_t* layout, int32_t layer_begin, int32_t layer_count,
                                  const void* q_raw, void* out, void* stream);
+
+/*
+ * ippd_read_probe -- measuring aid: enqueues a kernel that streams the key/value tiles of the step
+ * declared last, for `layer_count` layers, through the same bulk-copy ring, slices and grid as the
+ * tensor-core attention kernel and discards them (no tensor-core or softmax work, nothing written).
+ * Timed with events by the caller, it gives the read bandwidth attainable with the attention
+ * kernel's own access pattern.  Errors: IPPD_ERR_INVALID_ARG, IPPD_ERR_NOT_BOUND, IPPD_ERR_CUDA.
+ */
+int ippd_read_probe(ippd_layout_t* layout, int32_t layer_begin, int32_t layer_count, void* stream);
+
+/* Host time (microseconds, summed) spent inside ippd_begin_step -- planning the step, packing the
+ * branch tiles, staging the descriptor -- and the number of steps, since the last read.  Host-only. */
+int ippd_host_time_read(ippd_layout_t* layout, double* begin_step_us, int64_t* n_steps);
 
 /* Number of kernels this library has launched through this layout since it was built. */
 int64_t ippd_launch_count(const ippd_layout_t* layout);

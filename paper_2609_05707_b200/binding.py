@@ -25,8 +25,8 @@ APPEND_CONTEXT, APPEND_QUESTION, APPEND_STEP = 0, 1, 2
 OPT_KERNEL, OPT_LAYERS_PER_CALL, OPT_TILES_PER_SPLIT, OPT_WAIT_LIMIT_US, OPT_PROFILE = 1, 2, 3, 4, 5
 
 EXPORTS = ["ippd_build_layout", "ippd_layout_tables", "ippd_cache_bytes", "ippd_bind_cache", "ippd_set_option",
-           "ippd_begin_step", "ippd_step_descriptor_bytes", "ippd_append_kv", "ippd_workspace_bytes", "ippd_decode_attention", "ippd_decode_attention_static",
-           "ippd_decode_step_host", "ippd_decode_step_host_async", "ippd_host_steps_wait", "ippd_step_stage_bytes", "ippd_export_mask", "ippd_poll_status", "ippd_profile_read",
+           "ippd_begin_step", "ippd_step_descriptor_bytes", "ippd_append_kv", "ippd_workspace_bytes", "ippd_decode_attention", "ippd_decode_step", "ippd_decode_step_grouped", "ippd_decode_attention_static",
+           "ippd_decode_step_host", "ippd_decode_step_host_async", "ippd_host_steps_wait", "ippd_step_stage_bytes", "ippd_export_mask", "ippd_poll_status", "ippd_profile_read", "ippd_read_probe", "ippd_host_time_read",
            "ippd_launch_count", "ippd_last_error", "ippd_destroy_layout"]
 
 
@@ -58,6 +58,8 @@ lib.ippd_step_descriptor_bytes.argtypes = [_vp, _pi32, _pi32, _i32, C.POINTER(_s
 lib.ippd_append_kv.argtypes = [_vp, _i32, _i32, _i32, _pi32, _i32, _vp, _vp, _vp]
 lib.ippd_workspace_bytes.argtypes = [_vp, _i32, C.POINTER(_sz)]
 lib.ippd_decode_attention.argtypes = [_vp, _i32, _i32, _vp, _vp, _vp, _sz, _vp]
+lib.ippd_decode_step.argtypes = [_vp, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
+lib.ippd_decode_step_grouped.argtypes = [_vp, _i32, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
 lib.ippd_decode_attention_static.argtypes = [_vp, _i32, _i32, _vp, _vp, _vp]
 lib.ippd_decode_step_host.argtypes = [_vp, _pi32, _pi32, _i32, _vp, _vp, _vp, _vp, _vp, _sz, _vp, _sz, _vp]
 lib.ippd_decode_step_host_async.argtypes = [_vp, _pi32, _pi32, _i32, _vp, _vp, _vp, _vp, _vp, _sz, _vp, _sz, _vp]
@@ -67,6 +69,8 @@ lib.ippd_export_mask.argtypes = [_vp, _i32, _pi32, C.POINTER(C.c_uint8), C.POINT
 lib.ippd_poll_status.argtypes = [_vp, _pi32]
 lib.ippd_profile_read.argtypes = [_vp, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(C.c_double),
                                   C.POINTER(_i64)]
+lib.ippd_read_probe.argtypes = [_vp, _i32, _i32, _vp]
+lib.ippd_host_time_read.argtypes = [_vp, C.POINTER(C.c_double), C.POINTER(_i64)]
 lib.ippd_launch_count.argtypes = [_vp]
 lib.ippd_launch_count.restype = _i64
 lib.ippd_last_error.restype = C.c_char_p
@@ -180,6 +184,18 @@ class Layout:
         _check(lib.ippd_decode_attention(self._h, layer_begin, layer_count, _dev(q_raw), _dev(out), _dev(workspace),
                                          ws_bytes, stream), "ippd_decode_attention")
 
+    def decode_step(self, layer_begin: int, layer_count: int, q_raw, k_raw, v_raw, out, workspace, stream: int = 0):
+        """append_kv(STEP) + decode_attention in one launch."""
+        ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+        _check(lib.ippd_decode_step(self._h, layer_begin, layer_count, _dev(q_raw), _dev(k_raw), _dev(v_raw), _dev(out),
+                                    _dev(workspace), ws_bytes, stream), "ippd_decode_step")
+
+    def decode_step_grouped(self, layers_per_call: int, q_raw, k_raw, v_raw, out, workspace, stream: int = 0):
+        """decode_step for all layers of the step, `layers_per_call` layers per launch."""
+        ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+        _check(lib.ippd_decode_step_grouped(self._h, layers_per_call, _dev(q_raw), _dev(k_raw), _dev(v_raw), _dev(out),
+                                            _dev(workspace), ws_bytes, stream), "ippd_decode_step_grouped")
+
     def decode_attention_static(self, layer_begin: int, layer_count: int, q_raw, out, stream: int = 0):
         """Same result as decode_attention, for callers that may not allocate: the split-KV scratch is the
         library's built-in device array (STATIC_SCRATCH_BYTES per GPU) instead of a caller workspace."""
@@ -229,6 +245,14 @@ class Layout:
         a, m, p, n = C.c_double(), C.c_double(), C.c_double(), _i64()
         _check(lib.ippd_profile_read(self._h, C.byref(a), C.byref(m), C.byref(p), C.byref(n)), "ippd_profile_read")
         return {"attention_ms": a.value, "merge_ms": m.value, "append_ms": p.value, "n_attention": n.value}
+
+    def read_probe(self, layer_begin: int, layer_count: int, stream: int = 0):
+        _check(lib.ippd_read_probe(self._h, layer_begin, layer_count, stream), "ippd_read_probe")
+
+    def host_time_read(self) -> dict:
+        us, n = C.c_double(), _i64()
+        _check(lib.ippd_host_time_read(self._h, C.byref(us), C.byref(n)), "ippd_host_time_read")
+        return {"begin_step_us": us.value, "steps": n.value}
 
     def launch_count(self) -> int:
         return int(lib.ippd_launch_count(self._h))

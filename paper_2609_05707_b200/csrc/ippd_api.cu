@@ -1,14 +1,17 @@
 // C ABI of the IPPD library: device state, uploads, kernel launches.
 #include <cuda_runtime.h>
 
+#include <algorithm>
+#include <chrono>
 #include <cstdio>
 #include <cstring>
 #include <mutex>
 #include <new>
 
+#include "ippd_aux_kernels.cuh"
 #include "ippd_attn_mma.cuh"
 #include "ippd_attn_tc.cuh"
-#include "ippd_aux_kernels.cuh"
+#include "ippd_read_probe.cuh"
 #include "ippd_device.cuh"
 #include "ippd_internal.h"
 
@@ -22,7 +25,7 @@
   } while (0)
 
 static const int kRingSlots = 16;
-static const int kMaxCtas = 256;  // upper bound of the persistent kernel's grid (SM count)
+static const int kMaxCtas = IPPD_TC_MAX_CTAS;  // upper bound of the persistent kernel's grid (SM count)
 
 struct ippd_layout {
   IppdHostLayout h;
@@ -54,6 +57,8 @@ struct ippd_layout {
   int sm_count = 0;
   cudaStream_t last_stream = nullptr;
   int64_t launches = 0;
+  double host_plan_us = 0.0;  // host time spent in ippd_begin_step (planning, packing, staging) since the last read
+  int64_t host_plan_steps = 0;
   // optional event record: (kind, start, stop) per bracketed kernel; kind 0 attention, 1 merge, 2 append
   bool profile = false;        // the current step is bracketed
   int64_t profile_stride = 0;  // 0 off; N: every N-th step declared by ippd_begin_step is bracketed
@@ -339,8 +344,11 @@ static int ring_uploaded(ippd_layout* L, cudaStream_t stream) {
 static int ring_flush(ippd_layout* L, cudaStream_t stream) {
   if (L->pending_slot < 0) return IPPD_OK;
   const int slot = L->pending_slot;
-  ippd_upload_kernel<<<(L->pending_n16 + 255) / 256, 256, 0, stream>>>((const uint4*)L->ring_host_dev[slot],
-                                                                       (uint4*)L->ring_dev[slot], L->pending_n16);
+  // Programmatic launch: the copy touches only its own slot, so it runs while the kernel before it in the stream is
+  // still busy; the kernel waits for that predecessor only at its end, which keeps the stream's order for whatever
+  // comes next.
+  CUDA_TRY(launch_pdl(ippd_upload_kernel, dim3((L->pending_n16 + 255) / 256), dim3(256), 0, stream,
+                      (const uint4*)L->ring_host_dev[slot], (uint4*)L->ring_dev[slot], L->pending_n16));
   CUDA_TRY(cudaGetLastError());
   L->launches++;
   return ring_uploaded(L, stream);
@@ -359,6 +367,7 @@ extern "C" int ippd_begin_step(ippd_layout_t* L, const int32_t* active_q, const 
   if (!L) { ippd_set_error("ippd_begin_step: NULL layout"); return IPPD_ERR_INVALID_ARG; }
   if (!L->bound) { ippd_set_error("ippd_begin_step: no cache bound"); return IPPD_ERR_NOT_BOUND; }
   cudaStream_t stream = (cudaStream_t)stream_;
+  const auto host_t0 = std::chrono::steady_clock::now();
   L->have_step = false;
   L->profile = L->profile_stride > 0 && (L->profile_steps++ % L->profile_stride) == 0;
   int rc = ippd_host_plan_step(L->h, active_q, answer_idx, A, plan_layers(L), &L->plan);
@@ -405,6 +414,17 @@ extern "C" int ippd_begin_step(ippd_layout_t* L, const int32_t* active_q, const 
   for (const IppdRowBlock& rb : P.rbs) L->step_needs_merge |= rb.n_seg > 1;
   L->have_step = true;
   L->last_stream = stream;
+  L->host_plan_us += std::chrono::duration<double, std::micro>(std::chrono::steady_clock::now() - host_t0).count();
+  L->host_plan_steps++;
+  return IPPD_OK;
+}
+
+extern "C" int ippd_host_time_read(ippd_layout_t* L, double* begin_step_us, int64_t* n_steps) {
+  if (!L) { ippd_set_error("ippd_host_time_read: NULL layout"); return IPPD_ERR_INVALID_ARG; }
+  if (begin_step_us) *begin_step_us = L->host_plan_us;
+  if (n_steps) *n_steps = L->host_plan_steps;
+  L->host_plan_us = 0.0;
+  L->host_plan_steps = 0;
   return IPPD_OK;
 }
 
@@ -518,22 +538,45 @@ extern "C" int ippd_workspace_bytes(const ippd_layout_t* L, int32_t layer_count,
   return IPPD_OK;
 }
 
-// Grid of the persistent tensor-core kernel for `layer_count` layers of the current step.
-static void tc_partition(const ippd_layout* L, int layer_count, long long* total, long long* chunk, int* grid) {
+// Slices of the persistent tensor-core kernel for `layer_count` layers of the current step: fills a->total_tiles,
+// a->n_cta and a->cut; *any_partial tells whether a cut falls inside a row block's key sequence (then partials are
+// written and the merge kernel runs).
+static int tc_partition(const ippd_layout* L, int layer_count, IppdTcArgs* a, bool* any_partial) {
   const long long t1 = L->plan.total_tiles;
-  *total = t1 * L->h.geom.n_kv_heads * layer_count;
+  const long long total = t1 * L->h.geom.n_kv_heads * layer_count;
+  if (total >= INT32_MAX) { ippd_set_error("too many key tiles in one launch: pass fewer layers per call"); return IPPD_ERR_INVALID_ARG; }
   int n_cta = L->sm_count > 0 ? L->sm_count : 148;
   if (n_cta > kMaxCtas) n_cta = kMaxCtas;
-  long long ch = (*total + n_cta - 1) / n_cta;
-  if (L->h.opt_tiles_per_split > 0) ch = L->h.opt_tiles_per_split;  // test knob: forces cuts every `ch` tiles
+  long long ch = (total + n_cta - 1) / n_cta;
+  const bool forced = L->h.opt_tiles_per_split > 0;  // test knob: cuts every `ch` tiles, wherever they fall
+  if (forced) ch = L->h.opt_tiles_per_split;
   if (ch < 1) ch = 1;
-  long long g = (*total + ch - 1) / ch;
+  long long g = (total + ch - 1) / ch;
   if (g > n_cta) {  // more pieces than CTAs: grow the pieces
-    ch = (*total + n_cta - 1) / n_cta;
-    g = (*total + ch - 1) / ch;
+    ch = (total + n_cta - 1) / n_cta;
+    g = (total + ch - 1) / ch;
   }
-  *chunk = ch;
-  *grid = (int)g;
+  const std::vector<int32_t>& rbt = L->plan.rb_tile_begin;  // [n_rb + 1], rbt[n_rb] = t1
+  const long long slack = forced ? 0 : ch / 32;
+  *any_partial = false;
+  a->cut[0] = 0;
+  int n = 0;
+  for (long long c = 1; c <= g; ++c) {
+    long long x = std::min(total, c * ch);
+    if (x < total) {
+      const long long seq = x / t1, within = x - seq * t1;
+      size_t rb = std::upper_bound(rbt.begin(), rbt.end(), (int32_t)within) - rbt.begin() - 1;
+      const long long lower = seq * t1 + rbt[rb], upper = seq * t1 + rbt[rb + 1];
+      long long snapped = (x - lower <= upper - x) ? lower : upper;
+      if (std::llabs(snapped - x) <= slack && snapped > a->cut[n] && snapped < total) x = snapped;
+      if (x != lower && x != upper) *any_partial = true;
+    }
+    if (x <= a->cut[n]) continue;
+    a->cut[++n] = (int32_t)x;
+  }
+  a->total_tiles = (int)total;
+  a->n_cta = n;
+  return IPPD_OK;
 }
 
 // Bytes of scratch the current step needs for `layer_count` layers; *o_bytes = offset of the (m, l) part.
@@ -541,11 +584,11 @@ static size_t scratch_need(const ippd_layout* L, int layer_count, size_t* o_byte
   const IppdHostLayout& h = L->h;
   size_t n_part;
   if (h.kernel_path() == 2) {
-    long long total, chunk;
-    int grid;
-    tc_partition(L, layer_count, &total, &chunk, &grid);
-    n_part = (size_t)grid * 2 * IPPD_TC_ROWS;
-    *needed = grid > 1;
+    IppdTcArgs a;
+    bool any_partial = false;
+    if (tc_partition(L, layer_count, &a, &any_partial) != IPPD_OK) { a.n_cta = kMaxCtas; any_partial = true; }
+    n_part = (size_t)a.n_cta * 2 * IPPD_TC_ROWS;
+    *needed = any_partial;
   } else {
     n_part = (size_t)layer_count * h.geom.n_kv_heads * (size_t)L->step_dev.n_units * L->step_dev.RB;
     *needed = L->step_needs_merge;
@@ -556,7 +599,8 @@ static size_t scratch_need(const ippd_layout* L, int layer_count, size_t* o_byte
 
 template <int D>
 static int launch_attention(ippd_layout* L, const IppdDev& d, int layer_begin, int layer_count, const void* q_raw,
-                            void* out, float* part_o, float* part_ml, cudaStream_t stream, bool marks) {
+                            void* out, float* part_o, float* part_ml, cudaStream_t stream, bool marks,
+                            const void* k_step = nullptr, const void* v_step = nullptr) {
   {
     // once per device and head size; host threads making their first calls at the same time take turns
     static std::mutex mu;
@@ -576,8 +620,12 @@ static int launch_attention(ippd_layout* L, const IppdDev& d, int layer_begin, i
   int out_f32 = L->h.geom.out_dtype == IPPD_F32;
   if (L->h.kernel_path() == 2) {
     IppdTcArgs a;
-    int grid;
-    tc_partition(L, layer_count, &a.total_tiles, &a.chunk, &grid);
+    bool any_partial = false;
+    {
+      int rc = tc_partition(L, layer_count, &a, &any_partial);
+      if (rc != IPPD_OK) return rc;
+    }
+    const int grid = a.n_cta;
     a.rb_tile_begin = L->d_rb_tile_begin;
     a.tiles = L->d_tc_tiles;
     a.pieces = L->d_tc_pieces;
@@ -585,14 +633,16 @@ static int launch_attention(ippd_layout* L, const IppdDev& d, int layer_begin, i
     a.layer_begin = layer_begin;
     a.layer_count = layer_count;
     a.out_f32 = out_f32;
+    a.k_step = (const __nv_bfloat16*)k_step;
+    a.v_step = (const __nv_bfloat16*)v_step;
     if (marks) prof_mark(L, 0, true, stream);
     CUDA_TRY(launch_pdl(ippd_attn_tc_kernel<D>, dim3(grid), dim3(IPPD_TC_THREADS), (size_t)tc_smem_bytes<D>(), stream, d,
                         S, a, (const __nv_bfloat16*)q_raw, out, part_o, part_ml));
     if (marks) prof_mark(L, 0, false, stream);
     CUDA_TRY(cudaGetLastError());
     L->launches++;
-    if (grid > 1) {
-      dim3 mg((unsigned)S.n_rb * IPPD_TC_MERGE_SPLIT, (unsigned)Hkv, (unsigned)layer_count);
+    if (any_partial) {
+      dim3 mg((unsigned)(grid - 1) * IPPD_TC_MERGE_SPLIT);
       if (marks) prof_mark(L, 1, true, stream);
       CUDA_TRY(launch_pdl(ippd_merge_tc_kernel<D>, mg, dim3(128), 0, stream, d, S, a, (const float*)part_o,
                           (const float*)part_ml, out));
@@ -621,32 +671,41 @@ static int launch_attention(ippd_layout* L, const IppdDev& d, int layer_begin, i
   return IPPD_OK;
 }
 
-extern "C" int ippd_decode_attention(ippd_layout_t* L, int32_t layer_begin, int32_t layer_count, const void* q_raw,
-                                     void* out, void* workspace, size_t workspace_bytes, void* stream_) {
-  if (!L) { ippd_set_error("ippd_decode_attention: NULL layout"); return IPPD_ERR_INVALID_ARG; }
-  if (!L->bound) { ippd_set_error("ippd_decode_attention: no cache bound"); return IPPD_ERR_NOT_BOUND; }
-  if (!L->have_step) { ippd_set_error("ippd_decode_attention: call ippd_begin_step first"); return IPPD_ERR_INVALID_ARG; }
+// Common body of ippd_decode_attention (k_step == NULL) and ippd_decode_step.
+static int decode_attention_impl(ippd_layout_t* L, const char* who, int32_t layer_begin, int32_t layer_count,
+                                 const void* q_raw, const void* k_step, const void* v_step, void* out, void* workspace,
+                                 size_t workspace_bytes, void* stream_) {
+  const std::string name(who);
+  if (!L) { ippd_set_error(name + ": NULL layout"); return IPPD_ERR_INVALID_ARG; }
+  if (!L->bound) { ippd_set_error(name + ": no cache bound"); return IPPD_ERR_NOT_BOUND; }
+  if (!L->have_step) { ippd_set_error(name + ": call ippd_begin_step first"); return IPPD_ERR_INVALID_ARG; }
   const IppdHostLayout& h = L->h;
   if (layer_begin < 0 || layer_count < 1 || layer_begin + layer_count > h.geom.n_layers) {
-    ippd_set_error("ippd_decode_attention: layer range out of bounds");
+    ippd_set_error(name + ": layer range out of bounds");
     return IPPD_ERR_INVALID_ARG;
   }
   cudaStream_t stream = (cudaStream_t)stream_;
   L->last_stream = stream;
   const IppdStepDev& S = L->step_dev;
   if (S.A == 0) return IPPD_OK;
-  if (!q_raw || !out) { ippd_set_error("ippd_decode_attention: NULL q_raw / out"); return IPPD_ERR_INVALID_ARG; }
+  if (!q_raw || !out) { ippd_set_error(name + ": NULL q_raw / out"); return IPPD_ERR_INVALID_ARG; }
   size_t o_bytes = 0;
   bool needed = false;
   size_t need = scratch_need(L, layer_count, &o_bytes, &needed);
   float *part_o = nullptr, *part_ml = nullptr;
   if (needed) {
     if (!workspace || workspace_bytes < need || (uintptr_t)workspace % 256 != 0) {
-      ippd_set_error("ippd_decode_attention: workspace missing, misaligned or too small");
+      ippd_set_error(name + ": workspace missing, misaligned or too small");
       return IPPD_ERR_INVALID_ARG;
     }
     part_o = (float*)workspace;
     part_ml = (float*)((char*)workspace + o_bytes);
+  }
+  if (k_step && h.kernel_path() != 2) {
+    // the warp-level path has no append role: the step's tokens go through the append kernel first
+    int rc = ippd_append_kv(L, layer_begin, layer_count, IPPD_APPEND_STEP, nullptr, 0, k_step, v_step, stream_);
+    if (rc != IPPD_OK) return rc;
+    k_step = v_step = nullptr;
   }
   {
     int rc = ring_flush(L, stream);  // the step's descriptor, unless a STEP append carried it along
@@ -654,8 +713,25 @@ extern "C" int ippd_decode_attention(ippd_layout_t* L, int32_t layer_begin, int3
   }
   IppdDev d = make_dev(L);
   if (h.geom.head_dim == 128)
-    return launch_attention<128>(L, d, layer_begin, layer_count, q_raw, out, part_o, part_ml, stream, true);
-  return launch_attention<64>(L, d, layer_begin, layer_count, q_raw, out, part_o, part_ml, stream, true);
+    return launch_attention<128>(L, d, layer_begin, layer_count, q_raw, out, part_o, part_ml, stream, true, k_step, v_step);
+  return launch_attention<64>(L, d, layer_begin, layer_count, q_raw, out, part_o, part_ml, stream, true, k_step, v_step);
+}
+
+extern "C" int ippd_decode_attention(ippd_layout_t* L, int32_t layer_begin, int32_t layer_count, const void* q_raw,
+                                     void* out, void* workspace, size_t workspace_bytes, void* stream_) {
+  return decode_attention_impl(L, "ippd_decode_attention", layer_begin, layer_count, q_raw, nullptr, nullptr, out,
+                               workspace, workspace_bytes, stream_);
+}
+
+extern "C" int ippd_decode_step(ippd_layout_t* L, int32_t layer_begin, int32_t layer_count, const void* q_raw,
+                                const void* k_raw, const void* v_raw, void* out, void* workspace,
+                                size_t workspace_bytes, void* stream_) {
+  if (L && L->have_step && L->step_dev.A > 0 && (!k_raw || !v_raw)) {
+    ippd_set_error("ippd_decode_step: NULL k_raw / v_raw");
+    return IPPD_ERR_INVALID_ARG;
+  }
+  return decode_attention_impl(L, "ippd_decode_step", layer_begin, layer_count, q_raw, k_raw, v_raw, out, workspace,
+                               workspace_bytes, stream_);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -724,6 +800,71 @@ extern "C" int ippd_decode_attention_static(ippd_layout_t* L, int32_t layer_begi
   return launch_attention<64>(L, d, layer_begin, layer_count, q_raw, out, part_o, part_ml, stream, false);
 }
 
+extern "C" int ippd_decode_step_grouped(ippd_layout_t* L, int32_t layers_per_call, const void* q_raw, const void* k_raw,
+                                        const void* v_raw, void* out, void* workspace, size_t workspace_bytes,
+                                        void* stream_) {
+  if (!L) { ippd_set_error("ippd_decode_step_grouped: NULL layout"); return IPPD_ERR_INVALID_ARG; }
+  const ippd_geometry_t& g = L->h.geom;
+  if (layers_per_call < 1 || layers_per_call > g.n_layers) {
+    ippd_set_error("ippd_decode_step_grouped: bad layers_per_call");
+    return IPPD_ERR_INVALID_ARG;
+  }
+  const size_t A = L->have_step ? (size_t)L->step_dev.A : 0;
+  const size_t q_layer = A * g.n_q_heads * g.head_dim * 2, kv_layer = A * g.n_kv_heads * g.head_dim * 2;
+  const size_t o_layer = A * g.n_q_heads * g.head_dim * (g.out_dtype == IPPD_F32 ? 4 : 2);
+  for (int l0 = 0; l0 < g.n_layers; l0 += layers_per_call) {
+    const int n = std::min(layers_per_call, g.n_layers - l0);
+    int rc = ippd_decode_step(L, l0, n, (const char*)q_raw + l0 * q_layer, (const char*)k_raw + l0 * kv_layer,
+                              (const char*)v_raw + l0 * kv_layer, (char*)out + l0 * o_layer, workspace,
+                              workspace_bytes, stream_);
+    if (rc != IPPD_OK) return rc;
+  }
+  return IPPD_OK;
+}
+
+extern "C" int ippd_read_probe(ippd_layout_t* L, int32_t layer_begin, int32_t layer_count, void* stream_) {
+  if (!L) { ippd_set_error("ippd_read_probe: NULL layout"); return IPPD_ERR_INVALID_ARG; }
+  if (!L->bound) { ippd_set_error("ippd_read_probe: no cache bound"); return IPPD_ERR_NOT_BOUND; }
+  if (!L->have_step || L->h.kernel_path() != 2) {
+    ippd_set_error("ippd_read_probe: needs a step declared for the tensor-core path");
+    return IPPD_ERR_INVALID_ARG;
+  }
+  const IppdHostLayout& h = L->h;
+  if (layer_begin < 0 || layer_count < 1 || layer_begin + layer_count > h.geom.n_layers) {
+    ippd_set_error("ippd_read_probe: layer range out of bounds");
+    return IPPD_ERR_INVALID_ARG;
+  }
+  cudaStream_t stream = (cudaStream_t)stream_;
+  L->last_stream = stream;
+  if (L->step_dev.A == 0) return IPPD_OK;
+  int rc = ring_flush(L, stream);
+  if (rc != IPPD_OK) return rc;
+  IppdTcArgs a = {};
+  bool any_partial = false;
+  rc = tc_partition(L, layer_count, &a, &any_partial);
+  if (rc != IPPD_OK) return rc;
+  const int grid = a.n_cta;
+  a.rb_tile_begin = L->d_rb_tile_begin;
+  a.tiles = L->d_tc_tiles;
+  a.pieces = L->d_tc_pieces;
+  a.T1 = (int)L->plan.total_tiles;
+  a.layer_begin = layer_begin;
+  a.layer_count = layer_count;
+  IppdDev d = make_dev(L);
+  const int D = h.geom.head_dim;
+  const size_t smem = (size_t)IPPD_TC_NBUF * IPPD_TILE_TOKENS * D * 2 + IPPD_TC_NBUF * sizeof(uint64_t);
+  if (D == 128) {
+    CUDA_TRY(cudaFuncSetAttribute(ippd_read_probe_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    ippd_read_probe_kernel<128><<<grid, 64, smem, stream>>>(d, L->step_dev, a);
+  } else {
+    CUDA_TRY(cudaFuncSetAttribute(ippd_read_probe_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    ippd_read_probe_kernel<64><<<grid, 64, smem, stream>>>(d, L->step_dev, a);
+  }
+  CUDA_TRY(cudaGetLastError());
+  L->launches++;
+  return IPPD_OK;
+}
+
 extern "C" int ippd_step_stage_bytes(const ippd_layout_t* L, int32_t A, size_t* bytes) {
   if (!L || !bytes || A < 0) { ippd_set_error("ippd_step_stage_bytes: bad argument"); return IPPD_ERR_INVALID_ARG; }
   const ippd_geometry_t& g = L->h.geom;
@@ -762,9 +903,7 @@ extern "C" int ippd_decode_step_host(ippd_layout_t* L, const int32_t* active_q, 
   CUDA_TRY(cudaMemcpyAsync(dq, host_q, qb, cudaMemcpyHostToDevice, stream));
   CUDA_TRY(cudaMemcpyAsync(dk, host_k, kvb, cudaMemcpyHostToDevice, stream));
   CUDA_TRY(cudaMemcpyAsync(dv, host_v, kvb, cudaMemcpyHostToDevice, stream));
-  rc = ippd_append_kv(L, 0, g.n_layers, IPPD_APPEND_STEP, nullptr, 0, dk, dv, stream_);
-  if (rc != IPPD_OK) return rc;
-  rc = ippd_decode_attention(L, 0, g.n_layers, dq, dout, workspace, workspace_bytes, stream_);
+  rc = ippd_decode_step(L, 0, g.n_layers, dq, dk, dv, dout, workspace, workspace_bytes, stream_);
   if (rc != IPPD_OK) return rc;
   CUDA_TRY(cudaMemcpyAsync(host_out, dout, ob, cudaMemcpyDeviceToHost, stream));
   CUDA_TRY(cudaStreamSynchronize(stream));
@@ -825,9 +964,7 @@ extern "C" int ippd_decode_step_host_async(ippd_layout_t* L, const int32_t* acti
   if (rc != IPPD_OK) return rc;
   CUDA_TRY(cudaStreamWaitEvent(stream, L->hs_ev_in[slot], 0));
   if (reused) CUDA_TRY(cudaStreamWaitEvent(stream, L->hs_ev_out[slot], 0));
-  rc = ippd_append_kv(L, 0, g.n_layers, IPPD_APPEND_STEP, nullptr, 0, dk, dv, stream_);
-  if (rc != IPPD_OK) return rc;
-  rc = ippd_decode_attention(L, 0, g.n_layers, dq, dout, workspace, workspace_bytes, stream_);
+  rc = ippd_decode_step(L, 0, g.n_layers, dq, dk, dv, dout, workspace, workspace_bytes, stream_);
   if (rc != IPPD_OK) return rc;
   CUDA_TRY(cudaEventRecord(L->hs_ev_done[slot], stream));
   CUDA_TRY(cudaStreamWaitEvent(L->hs_out, L->hs_ev_done[slot], 0));

@@ -8,7 +8,7 @@
 // from the branches of several questions of the row block, laid one after the other (the host packs them per step);
 // a row may look only at the columns of its own question's piece -- the IPPD mask, realised structurally.
 //
-// Warp roles (608 threads):
+// Warp roles (640 threads):
 //   warp 0      producer: bulk async copies (TMA engine) of K and V into a 7-deep ring of 128-row buffers, mbarrier
 //               completion; only the 8-token groups that hold valid tokens are fetched.
 //   warp 1      P V issuer (one lane): O += P V with P read from TMEM (it overwrites the S buffer it came from) and V
@@ -22,25 +22,41 @@
 //               previous contents has completed.  Two issuers, because a tcgen05.mma holds its issuing thread about
 //               as long as it executes: one thread for both made a late K tile delay the P V products and a late P
 //               delay the S products.
+//   warp 19     append (only when the call carries the step's raw K/V): walks the CTA's slice ahead of the producer and,
+//               for every packed branch piece that holds the token fed at this step, rotates its key (RoPE) and writes
+//               K~ and V into the piece's cache slot; the producer fetches a packed tile only after its slots are in
+//               place.  A step's token belongs to exactly one piece of one (layer, KV head) sequence, so exactly one
+//               CTA writes it and only that CTA reads it in this launch.
 // Every wait is bounded; on expiry the error word is raised and all roles drain out.
 #pragma once
+#include "ippd_aux_kernels.cuh"
 #include "ippd_device.cuh"
 
-#define IPPD_TC_THREADS 608
+#define IPPD_TC_THREADS 640
+#define IPPD_TC_WARP_S_ISSUER 18
+#define IPPD_TC_WARP_APPEND 19
 #define IPPD_TC_NBUF 7
 #define IPPD_TC_ROWS 128
-#define IPPD_TC_MERGE_SPLIT 8  // merge blocks per (row block, KV head, layer)
+#define IPPD_TC_MERGE_SPLIT 8  // merge blocks per cut key sequence
+#define IPPD_TC_MAX_CTAS 192   // upper bound of the persistent grid (one CTA per SM)
 #define IPPD_TC_RESCALE_THRESHOLD 8.0f  // log2 units: the reference maximum may lag by up to 2^8
 
 struct IppdTcArgs {
   const int32_t* rb_tile_begin;  // [n_rb+1] first tile of each row block inside one (layer, head) sequence
   const IppdTcTile* tiles;       // [T1] tiles of one (layer, head) sequence
   const IppdTcPiece* pieces;     // pieces of the packed branch tiles
-  long long total_tiles;         // T1 * Hkv * layer_count
-  long long chunk;               // tiles per CTA
+  int total_tiles;               // T1 * Hkv * layer_count
+  int n_cta;                     // CTAs of the launch
+  // CTA c owns tiles [cut[c], cut[c+1]) of the launch's tile sequence.  The host cuts it into equal parts and moves a
+  // cut to the nearest boundary between two row blocks' key sequences when that is close: a sequence that is not cut
+  // needs no partial and no merge.
+  int32_t cut[IPPD_TC_MAX_CTAS + 1];
   int T1;                        // tiles of one (layer, head) sequence
   int layer_begin, layer_count;
   int out_f32;
+  // raw K and V of the step's tokens, [layer_count, A, Hkv, D] (pre-RoPE), when the call appends them itself; else NULL
+  const __nv_bfloat16* k_step;
+  const __nv_bfloat16* v_step;
 };
 
 // ---- tcgen05 wrappers ----
@@ -175,6 +191,7 @@ struct TcShared {
   uint64_t drain[2];     // completion of each issuer's MMAs in flight when it stops
   uint32_t tmem_base;
   volatile int abort_flag;
+  uint32_t app_done;     // the append warp has finished the packed tiles with index (in the CTA's slice) below this
   unsigned short xmax[2][4][IPPD_TC_ROWS];  // [tile parity][warpgroup][row]: bf16 bits of the quarter-row maxima
   TcMeta meta[IPPD_TC_NMETA];
 };
@@ -208,6 +225,29 @@ __device__ __forceinline__ bool tc_wait(uint64_t* bar, uint32_t parity, const Ip
   return true;
 }
 
+// Bounded wait until the append warp's progress counter has passed `need`.
+__device__ __forceinline__ bool tc_wait_appended(const uint32_t* counter, uint32_t need, const IppdDev& L, TcShared* sh) {
+  auto load = [&]() {
+    uint32_t v;
+    asm volatile("ld.acquire.cta.shared::cta.u32 %0, [%1];" : "=r"(v) : "r"(smem_u32(counter)) : "memory");
+    return v;
+  };
+  if (load() >= need) return true;
+  unsigned long long t0 = globaltimer_ns();
+  uint32_t spins = 0;
+  while (load() < need) {
+    if ((++spins & 63u) == 0) {
+      if (sh->abort_flag) return false;
+      if (globaltimer_ns() - t0 > (unsigned long long)L.wait_limit_ns) {
+        sh->abort_flag = 1;
+        atomicOr(L.error_word, IPPD_ERRBIT_TIMEOUT);
+        return false;
+      }
+    }
+  }
+  return true;
+}
+
 #include "ippd_attn_tc_softmax.cuh"
 
 template <int D>
@@ -224,8 +264,7 @@ ippd_attn_tc_kernel(IppdDev L, IppdStepDev S, IppdTcArgs A, const __nv_bfloat16*
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int Hkv = L.Hkv;
   pdl_trigger();  // the merge kernel may be scheduled as soon as SMs become free
-  const long long g0 = (long long)blockIdx.x * A.chunk;
-  const long long g1 = min(A.total_tiles, g0 + A.chunk);
+  const long long g0 = A.cut[blockIdx.x], g1 = A.cut[blockIdx.x + 1];
 
   if (tid == 0) {
     for (int i = 0; i < IPPD_TC_NBUF; ++i) { mbar_init(&sh->kv_full[i], 1); mbar_init(&sh->kv_empty[i], 1); }
@@ -236,6 +275,7 @@ ippd_attn_tc_kernel(IppdDev L, IppdStepDev S, IppdTcArgs A, const __nv_bfloat16*
     mbar_init(&sh->o_free, 16);
     mbar_init(&sh->q_full, 16);
     sh->abort_flag = 0;
+    sh->app_done = 0;
     mbar_fence_init();
   }
   if (warp == 1) {
@@ -277,6 +317,12 @@ ippd_attn_tc_kernel(IppdDev L, IppdStepDev S, IppdTcArgs A, const __nv_bfloat16*
                            ((uint32_t)pc.n_groups << 24);
         __syncwarp();
         const int groups = (ti.rows + 7) >> 3;
+        if (A.k_step != nullptr && ti.n_pieces > 0) {
+          // the step's own tokens are written by the append warp of this CTA: fetch the tile after them
+          if (lane == 0) ok = tc_wait_appended(&sh->app_done, tc + 1, L, sh);
+          ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+          if (!ok) break;
+        }
         for (int kv = 0; kv < 2 && ok; ++kv, ++n) {
           uint32_t buf = n % IPPD_TC_NBUF, ph = (n / IPPD_TC_NBUF) & 1;
           if (lane == 0) ok = tc_wait(&sh->kv_empty[buf], ph ^ 1, L, sh);
@@ -349,7 +395,57 @@ ippd_attn_tc_kernel(IppdDev L, IppdStepDev S, IppdTcArgs A, const __nv_bfloat16*
       tc_commit(&sh->drain[0]);
       mbar_wait_ns(&sh->drain[0], 0, L, IPPD_DRAIN_LIMIT_NS);
     }
-  } else if (warp == IPPD_TC_THREADS / 32 - 1) {
+  } else if (warp == IPPD_TC_WARP_APPEND) {
+    // =========================== append (RoPE + store of the step's tokens) ===========================
+    if (A.k_step != nullptr) {
+      constexpr int CP = D / 16;    // lanes per token: one per pair of 16-byte chunks (c, c + D/16)
+      constexpr int TPP = 32 / CP;  // tokens per pass of the warp
+      long long g = g0;
+      TcSegment sg;
+      uint32_t tc = 0;  // tiles of the slice passed so far (the producer counts the same way)
+      bool stop = false;
+      while (!stop && tc_next_segment(A, S, Hkv, g0, g1, g, sg)) {
+        const IppdRowBlock rb = S.rbs[sg.rb];
+        const int first_packed = A.rb_tile_begin[sg.rb] + rb.n_ctx_tiles;
+        const int layer = A.layer_begin + sg.ll;
+        for (int t = sg.t_begin; t < sg.t_end; ++t, ++tc) {
+          if (t < first_packed) continue;  // context tiles hold no token of this step
+          if (sh->abort_flag) { stop = true; break; }
+          const IppdTcTile ti = A.tiles[t];
+          IppdTcPiece pc;
+          pc.new_tok = 0;
+          if (lane < ti.n_pieces) pc = A.pieces[ti.piece_begin + lane];
+          unsigned todo = __ballot_sync(0xffffffffu, pc.new_tok != 0);
+          while (todo) {
+            // lane group gi takes the gi-th piece still to do
+            const int gi = lane / CP, c = lane % CP;
+            unsigned m = todo;
+            int src = 0;
+            for (int i = 0; i <= gi && m; ++i) { src = __ffs(m) - 1; m &= m - 1; }
+            const bool have = __popc(todo) > gi;
+            const int a_local = __shfl_sync(0xffffffffu, pc.a_local, src);
+            const int src_tile = __shfl_sync(0xffffffffu, pc.src_tile, src);
+            const int src_group = __shfl_sync(0xffffffffu, pc.src_group, src);
+            const int new_tok = __shfl_sync(0xffffffffu, pc.new_tok, src);
+            if (have) {
+              const int a = rb.act_begin + a_local;
+              const size_t row = (((size_t)sg.ll * S.A + a) * Hkv + sg.head) * D + c * 8;
+              ippd_rope_store_pair<D>(L, A.k_step + row, A.v_step + row, S.act_pos[a], c,
+                                      ippd_tile_addr(L, layer, sg.head, src_tile, 0), src_group * 8 + new_tok - 1);
+            }
+            for (int i = 0; i < TPP && todo; ++i) todo &= todo - 1;
+          }
+          // the stores above (generic proxy) are read by the producer's bulk copies (async proxy)
+          asm volatile("fence.proxy.async;" ::: "memory");
+          __syncwarp();
+          if (lane == 0)
+            asm volatile("st.release.cta.shared::cta.u32 [%0], %1;" ::"r"(smem_u32(&sh->app_done)), "r"(tc + 1) : "memory");
+        }
+      }
+      if (lane == 0)
+        asm volatile("st.release.cta.shared::cta.u32 [%0], %1;" ::"r"(smem_u32(&sh->app_done)), "r"(0xFFFFFFFFu) : "memory");
+    }
+  } else if (warp == IPPD_TC_WARP_S_ISSUER) {
     // =========================== S issuer (one lane) ===========================
     // S(j) = Q~ K(j)^T: Q~ from TMEM, K from ring slot 2j (K-major), into S buffer j & 1.  That buffer held P(j-2),
     // so PV(j-2) must have completed (pv_done): the two issuers' operations are not ordered by the tensor pipe.
@@ -407,20 +503,36 @@ ippd_attn_tc_kernel(IppdDev L, IppdStepDev S, IppdTcArgs A, const __nv_bfloat16*
 }
 
 // Log-sum-exp merge for the persistent kernel: a row block whose key sequence was cut across CTAs has one partial
-// per CTA that touched it (slot 0 if the piece is that CTA's first segment, else slot 1).
+// per CTA that touched it (slot 0 if the piece is that CTA's first segment, else slot 1).  Blocks [c * SPLIT,
+// (c + 1) * SPLIT) look at interior cut c + 1: if it falls strictly inside a key sequence and is the first cut to do so,
+// they merge that sequence's partials; otherwise they have nothing to do.
 template <int D>
 __global__ void __launch_bounds__(128)
 ippd_merge_tc_kernel(IppdDev L, IppdStepDev S, IppdTcArgs A, const float* __restrict__ part_o,
                      const float* __restrict__ part_ml, void* __restrict__ out) {
   pdl_trigger();
   pdl_wait();
-  const int rbi = blockIdx.x / IPPD_TC_MERGE_SPLIT, part = blockIdx.x % IPPD_TC_MERGE_SPLIT;
+  const int ci = blockIdx.x / IPPD_TC_MERGE_SPLIT + 1, part = blockIdx.x % IPPD_TC_MERGE_SPLIT;
+  const int x = A.cut[ci];
+  const int seq = x / A.T1, within = x - seq * A.T1;
+  int rbi = 0;
+  {
+    int lo = 0, hi = S.n_rb - 1;
+    while (lo < hi) {
+      int mid = (lo + hi + 1) >> 1;
+      if (A.rb_tile_begin[mid] <= within) lo = mid; else hi = mid - 1;
+    }
+    rbi = lo;
+  }
+  const int a0 = seq * A.T1 + A.rb_tile_begin[rbi];
+  if (x == a0) return;              // the cut sits between two key sequences
+  if (A.cut[ci - 1] > a0) return;   // an earlier cut lies inside the same sequence: its blocks do the merge
   const IppdRowBlock rb = S.rbs[rbi];
-  const int head = blockIdx.y, ll = blockIdx.z, G = L.G;
-  const long long a0 = ((long long)ll * L.Hkv + head) * A.T1 + A.rb_tile_begin[rbi];
-  const long long b0 = a0 + rb.n_tiles;
-  const long long c0 = a0 / A.chunk, c1 = (b0 - 1) / A.chunk;
-  if (c0 == c1) return;  // written directly by the one CTA that held the whole sequence
+  const int ll = seq / L.Hkv, head = seq - ll * L.Hkv, G = L.G;
+  const int b0 = a0 + rb.n_tiles;
+  const int c0 = ci - 1;  // the CTA that holds the sequence's first tiles
+  int c1 = ci;            // ... and the one that holds its last tile
+  while (c1 + 1 < A.n_cta && A.cut[c1 + 1] < b0) ++c1;
   const int nrows = rb.n_act * G;
   for (int item = part * blockDim.x + threadIdx.x; item < nrows * (D / 4); item += blockDim.x * IPPD_TC_MERGE_SPLIT) {
     int r = item / (D / 4), cc = item - r * (D / 4);
@@ -429,8 +541,8 @@ ippd_merge_tc_kernel(IppdDev L, IppdStepDev S, IppdTcArgs A, const float* __rest
     float M = -INFINITY, lsum = 0.f;
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll 2
-    for (long long c = c0; c <= c1; ++c) {
-      const size_t slot = (size_t)c * 2 + ((c * A.chunk >= a0) ? 0 : 1);
+    for (int c = c0; c <= c1; ++c) {
+      const size_t slot = (size_t)c * 2 + ((A.cut[c] >= a0) ? 0 : 1);
       const float2 ml = *reinterpret_cast<const float2*>(part_ml + (slot * IPPD_TC_ROWS + r) * 2);
       const float4 v = *reinterpret_cast<const float4*>(part_o + (slot * IPPD_TC_ROWS + r) * D + cc * 4);
       if (ml.x == -INFINITY) continue;  // this part of the key sequence held nothing the row may see

@@ -14,6 +14,56 @@ __global__ void ippd_rope_table_kernel(float2* table, int max_pos, int D, double
   table[idx] = make_float2((float)c, (float)s);
 }
 
+// RoPE + store of one (token, KV head, pair of 16-byte chunks c and c + D/16): the two halves of 8 rotation pairs of K,
+// and the same two chunks of V.  k_src / v_src point at chunk c of the token's raw row; `k_tile` is the byte offset of
+// the K half of the destination cache tile (its V half follows it), `u` the token's row inside the tile.  Cache tile
+// layout (K and V alike): [token/8][d/8][token%8][d%8] bf16, i.e. 8x8 blocks of 128 contiguous bytes.
+template <int D>
+__device__ __forceinline__ void ippd_rope_store_pair(const IppdDev& L, const __nv_bfloat16* __restrict__ k_src,
+                                                     const __nv_bfloat16* __restrict__ v_src, int pos, int c,
+                                                     size_t k_tile, int u) {
+  constexpr int CP = D / 16;
+  constexpr int GB = (D / 8) * 128;
+  uint4 klo = *reinterpret_cast<const uint4*>(k_src);
+  uint4 khi = *reinterpret_cast<const uint4*>(k_src + D / 2);
+  uint4 vlo = *reinterpret_cast<const uint4*>(v_src);
+  uint4 vhi = *reinterpret_cast<const uint4*>(v_src + D / 2);
+  {
+    // A NaN or an infinity (bf16: all exponent bits set) is stored like any value but reported: a cache row shares
+    // its 128-row tile with rows of other questions, and 0 x NaN would reach their outputs too.
+    const uint32_t* w[4] = {reinterpret_cast<const uint32_t*>(&klo), reinterpret_cast<const uint32_t*>(&khi),
+                            reinterpret_cast<const uint32_t*>(&vlo), reinterpret_cast<const uint32_t*>(&vhi)};
+    bool bad = false;
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+      for (int e = 0; e < 4; ++e)
+        bad |= (w[i][e] & 0x7F800000u) == 0x7F800000u || (w[i][e] & 0x00007F80u) == 0x00007F80u;
+    if (bad) atomicOr(L.error_word, IPPD_ERRBIT_NONFINITE);
+  }
+  const float2* cs = L.rope + (size_t)pos * (D / 2) + c * 8;
+  const __nv_bfloat162* pl = reinterpret_cast<const __nv_bfloat162*>(&klo);
+  const __nv_bfloat162* ph = reinterpret_cast<const __nv_bfloat162*>(&khi);
+  uint4 olo, ohi;
+  uint32_t* wl = reinterpret_cast<uint32_t*>(&olo);
+  uint32_t* wh = reinterpret_cast<uint32_t*>(&ohi);
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    float2 c0 = cs[2 * e], c1 = cs[2 * e + 1];
+    float l0 = __bfloat162float(pl[e].x), l1 = __bfloat162float(pl[e].y);
+    float h0 = __bfloat162float(ph[e].x), h1 = __bfloat162float(ph[e].y);
+    wl[e] = pack_bf16(l0 * c0.x - h0 * c0.y, l1 * c1.x - h1 * c1.y);
+    wh[e] = pack_bf16(h0 * c0.x + l0 * c0.y, h1 * c1.x + l1 * c1.y);
+  }
+  const size_t in_tile = (size_t)(u >> 3) * GB + (size_t)(u & 7) * 16;
+  char* kdst = L.cache + k_tile + in_tile;
+  char* vdst = kdst + (size_t)IPPD_TILE_TOKENS * D * 2;  // the V half of the tile follows its K half
+  *reinterpret_cast<uint4*>(kdst + c * 128) = olo;
+  *reinterpret_cast<uint4*>(kdst + (c + CP) * 128) = ohi;
+  *reinterpret_cast<uint4*>(vdst + c * 128) = vlo;
+  *reinterpret_cast<uint4*>(vdst + (c + CP) * 128) = vhi;
+}
+
 #define IPPD_APPEND_INLINE 64
 
 struct IppdAppendArgs {
@@ -33,15 +83,12 @@ struct IppdAppendArgs {
   int32_t act_q[IPPD_APPEND_INLINE], act_s[IPPD_APPEND_INLINE];
 };
 
-// One thread moves one (token, KV head, pair of 16-byte chunks c and c + D/16): the two halves of
-// 8 RoPE pairs of K, and the same two chunks of V.  Cache tile layout (K and V alike):
-// [token/8][d/8][token%8][d%8] bf16, i.e. 8x8 blocks of 128 contiguous bytes.
+// One thread moves one (token, KV head, pair of 16-byte chunks c and c + D/16), see ippd_rope_store_pair.
 template <int D>
 __global__ void __launch_bounds__(256)
 ippd_append_kernel(IppdDev L, IppdStepDev S, IppdAppendArgs a, int layer_begin,
                    const __nv_bfloat16* __restrict__ k_raw, const __nv_bfloat16* __restrict__ v_raw) {
   constexpr int CP = D / 16;  // chunk pairs per row
-  constexpr int GB = (D / 8) * 128;
   pdl_trigger();
   pdl_wait();
   if (a.n_append_blocks > 0 && (int)blockIdx.x >= a.n_append_blocks) {
@@ -89,44 +136,7 @@ ippd_append_kernel(IppdDev L, IppdStepDev S, IppdAppendArgs a, int layer_begin,
     return;
   }
   size_t src = (((size_t)ll * a.n_tokens + tok) * L.Hkv + head) * D + c * 8;
-  uint4 klo = *reinterpret_cast<const uint4*>(k_raw + src);
-  uint4 khi = *reinterpret_cast<const uint4*>(k_raw + src + D / 2);
-  uint4 vlo = *reinterpret_cast<const uint4*>(v_raw + src);
-  uint4 vhi = *reinterpret_cast<const uint4*>(v_raw + src + D / 2);
-  {
-    // A NaN or an infinity (bf16: all exponent bits set) is stored like any value but reported: a cache row shares
-    // its 128-row tile with rows of other questions, and 0 x NaN would reach their outputs too.
-    const uint32_t* w[4] = {reinterpret_cast<const uint32_t*>(&klo), reinterpret_cast<const uint32_t*>(&khi),
-                            reinterpret_cast<const uint32_t*>(&vlo), reinterpret_cast<const uint32_t*>(&vhi)};
-    bool bad = false;
-#pragma unroll
-    for (int i = 0; i < 4; ++i)
-#pragma unroll
-      for (int e = 0; e < 4; ++e)
-        bad |= (w[i][e] & 0x7F800000u) == 0x7F800000u || (w[i][e] & 0x00007F80u) == 0x00007F80u;
-    if (bad) atomicOr(L.error_word, IPPD_ERRBIT_NONFINITE);
-  }
-  const float2* cs = L.rope + (size_t)pos * (D / 2) + c * 8;
-  const __nv_bfloat162* pl = reinterpret_cast<const __nv_bfloat162*>(&klo);
-  const __nv_bfloat162* ph = reinterpret_cast<const __nv_bfloat162*>(&khi);
-  uint4 olo, ohi;
-  uint32_t* wl = reinterpret_cast<uint32_t*>(&olo);
-  uint32_t* wh = reinterpret_cast<uint32_t*>(&ohi);
-#pragma unroll
-  for (int e = 0; e < 4; ++e) {
-    float2 c0 = cs[2 * e], c1 = cs[2 * e + 1];
-    float l0 = __bfloat162float(pl[e].x), l1 = __bfloat162float(pl[e].y);
-    float h0 = __bfloat162float(ph[e].x), h1 = __bfloat162float(ph[e].y);
-    wl[e] = pack_bf16(l0 * c0.x - h0 * c0.y, l1 * c1.x - h1 * c1.y);
-    wh[e] = pack_bf16(h0 * c0.x + l0 * c0.y, h1 * c1.x + l1 * c1.y);
-  }
-  size_t in_tile = (size_t)(u >> 3) * GB + (size_t)(u & 7) * 16;
-  char* kdst = L.cache + ippd_tile_addr(L, layer, head, tile, 0) + in_tile;
-  char* vdst = L.cache + ippd_tile_addr(L, layer, head, tile, 1) + in_tile;
-  *reinterpret_cast<uint4*>(kdst + c * 128) = olo;
-  *reinterpret_cast<uint4*>(kdst + (c + CP) * 128) = ohi;
-  *reinterpret_cast<uint4*>(vdst + c * 128) = vlo;
-  *reinterpret_cast<uint4*>(vdst + (c + CP) * 128) = vhi;
+  ippd_rope_store_pair<D>(L, k_raw + src, v_raw + src, pos, c, ippd_tile_addr(L, layer, head, tile, 0), u);
 }
 
 // Token descriptor of the mask export: kind 0 = context token, 1 = question token, 2 = answer token.
@@ -157,9 +167,14 @@ __global__ void ippd_export_mask_kernel(IppdDev L, const IppdMaskTok* toks, int 
   out[idx] = ok ? 1 : 0;
 }
 
-// Copies a step descriptor from pinned host memory (read through its device mapping) to device memory.
+// Copies a step descriptor from pinned host memory (read through its device mapping) to device memory.  Launched
+// programmatically: nothing it touches depends on the kernel before it in the stream (the host wrote the pinned slot
+// before the launch, and the device slot's previous readers finished long ago), so the copy runs first and the wait
+// for that kernel comes last -- it only keeps the stream's order for the kernels that follow.
 __global__ void __launch_bounds__(256) ippd_upload_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst,
                                                           unsigned n16) {
+  pdl_trigger();
   const unsigned i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i < n16) dst[i] = src[i];
+  pdl_wait();
 }

@@ -193,7 +193,8 @@ int ippd_host_plan_step(const IppdHostLayout& L, const int32_t* active_q, const 
         const int G = L.geom.n_q_heads / L.geom.n_kv_heads;
         const int q_per_quarter = std::max(1, 32 / G);
         const int n_quarters = (rb.n_act + q_per_quarter - 1) / q_per_quarter;
-        struct Run { int a, cache_tile, off, groups, valid; };  // 8-token groups [off, off+groups) of one cache tile
+        // 8-token groups [off, off+groups) of one cache tile; `last`: the tile that holds the branch's newest token
+        struct Run { int a, cache_tile, off, groups, valid, last; };
         static thread_local std::vector<Run> runs[4];
         size_t next[4] = {0, 0, 0, 0};
         int rem[4] = {0, 0, 0, 0};  // groups each quarter still has to place
@@ -206,7 +207,8 @@ int ippd_host_plan_step(const IppdHostLayout& L, const int32_t* active_q, const 
             const int len = L.q_len[k] + answer_idx[a] + 1;
             for (int jt = 0; jt * IPPD_TILE_TOKENS < len; ++jt) {
               const int valid_j = std::min(IPPD_TILE_TOKENS, len - jt * IPPD_TILE_TOKENS);
-              runs[qu].push_back({a - a0, L.branch_tile_off[k] + jt, 0, (valid_j + 7) / 8, valid_j});
+              runs[qu].push_back({a - a0, L.branch_tile_off[k] + jt, 0, (valid_j + 7) / 8, valid_j,
+                                  (jt + 1) * IPPD_TILE_TOKENS >= len});
               rem[qu] += (valid_j + 7) / 8;
             }
           }
@@ -238,6 +240,9 @@ int ippd_host_plan_step(const IppdHostLayout& L, const int32_t* active_q, const 
               Run& r = runs[qu][next[qu]];
               const int take = std::min(want, r.groups);
               IppdTcPiece pc = {r.a, r.cache_tile, r.off, take, used * 8, std::min(take * 8, r.valid - r.off * 8), 0, 0};
+              // the token fed at this step is the branch's last valid token: exactly one piece of the step holds it
+              const int newest = r.valid - 1 - r.off * 8;
+              if (r.last && newest >= 0 && newest < take * 8) pc.new_tok = 1 + newest;
               plan->tc_pieces.push_back(pc);
               ti.n_pieces++;
               used += take;

@@ -53,7 +53,8 @@ struct IppdTcPiece {
   int32_t n_groups;
   int32_t row0;       // first row in the packed tile (multiple of 8)
   int32_t valid;      // valid tokens in the piece (<= 8 * n_groups)
-  int32_t pad0, pad1;
+  int32_t new_tok;    // 1 + index inside the piece of the token fed at this step, 0 if the piece does not hold it
+  int32_t pad1;
 };
 
 struct IppdStepPlan {

@@ -18,10 +18,12 @@ from .workloads import Workload
 
 class Runner:
     def __init__(self, wl: Workload, device: str = "cuda:0", out_dtype: int = B.BF16, kernel: int = 0,
-                 layers_per_call: Optional[int] = None, tiles_per_split: int = 0, branch_align: int = B.TILE_TOKENS):
+                 layers_per_call: Optional[int] = None, tiles_per_split: int = 0, branch_align: int = B.TILE_TOKENS,
+                 fused: bool = True):
         if not torch.cuda.is_available():
             raise RuntimeError("the IPPD library needs a CUDA device; there is no CPU fallback")
         self.wl = wl
+        self.fused = fused  # one ippd_decode_step call per layer group instead of append_kv(STEP) + decode_attention
         self.device = torch.device(device)
         torch.cuda.set_device(self.device)
         g = wl.geom
@@ -89,11 +91,39 @@ class Runner:
         if A == 0:
             return out
         lpc = self.layers_per_call
+        if self.fused:
+            self.layout.decode_step_grouped(lpc, q, k, v, out, self.workspace, self.stream)
+            return out
         for l0 in range(0, g.n_layers, lpc):
             n = min(lpc, g.n_layers - l0)
             self.layout.append_kv(l0, n, B.APPEND_STEP, None, k[l0:l0 + n], v[l0:l0 + n], self.stream)
             self.layout.decode_attention(l0, n, q[l0:l0 + n], out[l0:l0 + n], self.workspace, self.stream)
         return out
+
+    def set_layers_per_call(self, n: int):
+        """Changes the number of layers per launch (the next begin_step plans for it; the workspace is re-sized)."""
+        self.layout.set_option(B.OPT_LAYERS_PER_CALL, n)
+        self.layers_per_call = n
+        need = self.layout.workspace_bytes(n)
+        if need > self.workspace.numel():
+            self.workspace = self.alloc_bytes(need, "workspace")
+
+    def append_all_steps(self, layers_per_chunk: int = 8):
+        """Writes the K/V of EVERY decode step of the schedule into the cache (a step's slot depends only on the
+        question and the step index), so that afterwards any step can be run in any order."""
+        wl, g = self.wl, self.wl.geom
+        for s in range(wl.n_steps):
+            act = wl.active(s)
+            if len(act) == 0:
+                continue
+            self.layout.begin_step(act, np.full(len(act), s, dtype=np.int32), self.stream)
+            for l0 in range(0, g.n_layers, layers_per_chunk):
+                n = min(layers_per_chunk, g.n_layers - l0)
+                kv = [wl.step_kv(s, l, act, self.device) for l in range(l0, l0 + n)]
+                k = torch.stack([a for a, _ in kv]).contiguous()
+                v = torch.stack([b for _, b in kv]).contiguous()
+                self.layout.append_kv(l0, n, B.APPEND_STEP, None, k, v, self.stream)
+            torch.cuda.synchronize(self.device)
 
     def run_step(self, s: int):
         """Generates the inputs of workload step s and runs it; returns (active ids, out)."""

@@ -82,8 +82,13 @@ def _steps(wl, extra=()):
     return sorted({0, last, *before_eos, *extra})
 
 
-@pytest.mark.parametrize("kernel", [2, 1])
-def test_c2_full_size_sampled(kernel):
+def test_c2_full_size_sampled_warp_level_path():
+    # the earlier mma.sync path (IPPD_OPT_KERNEL = 1) on a thinner sample
+    lh = [(0, 0), (17, 5), (31, 7)]
+    run_and_sample("C2", {0: lh, 40: lh}, per_prompt=16, kernel=1)
+
+
+def test_c2_full_size_sampled(kernel=2):
     wl = W.make_workload("C2")
     # C2 has no stop steps: four steps spread over the schedule; every KV head of layer 17 at step 63 (= every tuple
     # of that layer and step)

@@ -160,3 +160,25 @@ def test_bf16_output_and_256_token_branch_alignment(kernel):
     cache = {}
     for s in range(wl.n_steps):
         compare_step(run, s, [0, 1], range(2), cache, "bf16 out, align 256")
+
+
+@pytest.mark.parametrize("tiles_per_split", [0, 3, 1000])
+def test_one_launch_step_equals_append_then_attention_bit_for_bit(tiles_per_split):
+    # ippd_decode_step writes the step's K~/V from inside the attention kernel; the cache and the outputs must be the
+    # ones ippd_append_kv(STEP) + ippd_decode_attention produce (same tiles, same arithmetic: bitwise), for whole
+    # sequences per CTA, for the library's own split and for cuts every three tiles (branch tiles cut from their
+    # context, tokens of one branch appended by different CTAs)
+    base = _base()
+    res = []
+    for fused in (False, True):
+        run = PoisonedRunner(base, out_dtype=B.F32, tiles_per_split=tiles_per_split, fused=fused, layers_per_call=1)
+        run.load_header()
+        outs = []
+        for s in range(base.n_steps):
+            act, out = run.run_step(s)
+            run.check()
+            outs.append(out.clone())
+        res.append((outs, run.cache.clone()))
+    for a, b in zip(res[0][0], res[1][0]):
+        assert torch.equal(a, b)
+    assert torch.equal(res[0][1], res[1][1])
