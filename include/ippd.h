@@ -338,7 +338,8 @@ int ippd_decode_attention_static(ippd_layout_t* layout, int32_t layer_begin, int
 int ippd_read_probe(ippd_layout_t* layout, int32_t layer_begin, int32_t layer_count, void* stream);
 
 /* Host time (microseconds, summed) spent inside ippd_begin_step -- planning the step, packing the
- * branch tiles, staging the descriptor -- and the number of steps, since the last read.  Host-only. */
+ * branch tiles, staging the descriptor; waiting for a free staging slot while the device is behind
+ * is not counted -- and the number of steps, since the last read.  Host-only. */
 int ippd_host_time_read(ippd_layout_t* layout, double* begin_step_us, int64_t* n_steps);
 
 /* Number of kernels this library has launched through this layout since it was built. */

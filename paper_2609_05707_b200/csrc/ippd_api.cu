@@ -58,6 +58,7 @@ struct ippd_layout {
   cudaStream_t last_stream = nullptr;
   int64_t launches = 0;
   double host_plan_us = 0.0;  // host time spent in ippd_begin_step (planning, packing, staging) since the last read
+  double host_wait_us = 0.0;  // part of it spent waiting for a free staging slot (the device is behind)
   int64_t host_plan_steps = 0;
   // optional event record: (kind, start, stop) per bracketed kernel; kind 0 attention, 1 merge, 2 append
   bool profile = false;        // the current step is bracketed
@@ -320,7 +321,12 @@ static int ring_stage(ippd_layout* L, const void* blob, size_t bytes, char** dev
   if (bytes > L->ring_cap) { ippd_set_error("descriptor larger than the staging slot"); return IPPD_ERR_CAPACITY; }
   int slot = L->ring_next;
   L->ring_next = (L->ring_next + 1) % kRingSlots;
-  if (L->ring_used[slot]) CUDA_TRY(cudaEventSynchronize(L->ring_ev[slot]));
+  if (L->ring_used[slot]) {
+    // back-pressure, not work: the host may run at most kRingSlots descriptors ahead of the device
+    const auto w0 = std::chrono::steady_clock::now();
+    CUDA_TRY(cudaEventSynchronize(L->ring_ev[slot]));
+    L->host_wait_us += std::chrono::duration<double, std::micro>(std::chrono::steady_clock::now() - w0).count();
+  }
   memcpy(L->ring_host[slot], blob, bytes);
   L->pending_slot = slot;
   L->pending_n16 = (unsigned)((bytes + 15) / 16);
@@ -421,7 +427,8 @@ extern "C" int ippd_begin_step(ippd_layout_t* L, const int32_t* active_q, const 
 
 extern "C" int ippd_host_time_read(ippd_layout_t* L, double* begin_step_us, int64_t* n_steps) {
   if (!L) { ippd_set_error("ippd_host_time_read: NULL layout"); return IPPD_ERR_INVALID_ARG; }
-  if (begin_step_us) *begin_step_us = L->host_plan_us;
+  if (begin_step_us) *begin_step_us = L->host_plan_us - L->host_wait_us;
+  L->host_wait_us = 0.0;
   if (n_steps) *n_steps = L->host_plan_steps;
   L->host_plan_us = 0.0;
   L->host_plan_steps = 0;

@@ -174,13 +174,15 @@ __device__ __forceinline__ bool tc_next_segment(const IppdTcArgs& a, const IppdS
   return true;
 }
 
-#define IPPD_TC_NMETA 8
-// Per-tile description staged in shared memory by the producer warp (it runs at most 4 tiles ahead of the softmax
-// warps).  piece[i] = a_local | row0 << 8 | valid << 16 | n_groups << 24.
+#define IPPD_TC_NMETA 5
+// Per-tile description staged in shared memory by the producer warp.  The producer starts tile t + 5 only after the
+// P V product of tile t has released its V buffer (7 ring buffers, two per tile), and every reader of tile t's entry
+// is done by then, so five entries suffice.  For a packed branch tile, [c0[a], c1[a]) are the columns question `a` of
+// the row block owns in it (the union of its adjacent pieces; empty when it has none).
 struct TcMeta {
   int32_t rows;
   int32_t n_pieces;
-  uint32_t piece[16];
+  uint8_t c0[64], c1[64];
 };
 
 struct TcShared {
@@ -312,9 +314,19 @@ ippd_attn_tc_kernel(IppdDev L, IppdStepDev S, IppdTcArgs A, const __nv_bfloat16*
         if (lane < ti.n_pieces) pc = A.pieces[ti.piece_begin + lane];
         TcMeta& mt = sh->meta[tc % IPPD_TC_NMETA];
         if (lane == 0) { mt.rows = ti.rows; mt.n_pieces = ti.n_pieces; }
-        if (lane < ti.n_pieces)
-          mt.piece[lane] = (uint32_t)pc.a_local | ((uint32_t)pc.row0 << 8) | ((uint32_t)pc.valid << 16) |
-                           ((uint32_t)pc.n_groups << 24);
+        if (ti.n_pieces > 0) {
+          // column window of every question in this tile: its pieces sit on adjacent lanes, the first gives c0 and
+          // the last c1 (only the last piece of a question can be partly valid)
+          reinterpret_cast<uint32_t*>(mt.c0)[lane & 15] = 0u;  // 64 + 64 bytes: lanes 0..15 clear c0, 16..31 clear c1
+          if (lane >= 16) reinterpret_cast<uint32_t*>(mt.c1)[lane & 15] = 0u;
+          __syncwarp();
+          const int a_me = lane < ti.n_pieces ? pc.a_local : -1;
+          const int a_prev = __shfl_up_sync(0xffffffffu, a_me, 1), a_next = __shfl_down_sync(0xffffffffu, a_me, 1);
+          if (lane < ti.n_pieces) {
+            if (lane == 0 || a_prev != a_me) mt.c0[a_me] = (uint8_t)pc.row0;
+            if (lane == ti.n_pieces - 1 || a_next != a_me) mt.c1[a_me] = (uint8_t)(pc.row0 + pc.valid);
+          }
+        }
         __syncwarp();
         const int groups = (ti.rows + 7) >> 3;
         if (A.k_step != nullptr && ti.n_pieces > 0) {

@@ -174,18 +174,9 @@ __device__ __forceinline__ void tc_softmax_role(const IppdDev& L, const IppdStep
           if (n_pieces == 0) {
             c1 = tile_rows;
           } else {
-            // a question may have two pieces in one tile (the end of one 128-token cache tile and the start of the
-            // next); they are adjacent and only the last one can be partly valid, so their union is one interval
-            bool found = false;
-            for (int pi = 0; pi < n_pieces; ++pi) {
-              const uint32_t pw = meta.piece[pi];
-              if ((int)(pw & 0xFF) == my_q) {
-                const int r0 = (pw >> 8) & 0xFF;
-                if (!found) c0 = r0;
-                found = true;
-                c1 = r0 + ((pw >> 16) & 0xFF);
-              }
-            }
+            // the producer has reduced the tile's pieces to one column window per question
+            c0 = meta.c0[my_q];
+            c1 = meta.c1[my_q];
           }
         }
         lo = min(IPPD_TC_CW, max(0, c0 - base));
