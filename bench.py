@@ -428,6 +428,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-layer-modes", action="store_true")
+    ap.add_argument("--sweep", action="store_true",
+                    help="questions-per-context x context-length table (the SWEEP-L*-Q* workloads) instead of the headline line")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
@@ -465,6 +467,24 @@ def main():
         if world > 1:
             dist.barrier()
             torch.cuda.synchronize()
+
+    if args.sweep:
+        # the axes of the paper's ablations: one JSON line holding the whole table
+        from paper_2609_05707_b200 import workloads as W2
+        args.no_layer_modes = True
+        rows = []
+        for L in W2.SWEEP_CONTEXTS:
+            for Q in W2.SWEEP_QUESTIONS:
+                e, c, _ = measure_config(f"SWEEP-L{L}-Q{Q}", args, dev, peaks, sync_all, False, 1)
+                c.close()
+                r = e["roofline"]
+                rows.append({"context": L, "questions": Q, "ms_per_step": e["ms_per_step"], "value": e["value"],
+                             "call_us": r["avg_call_us"], "hbm_gbs": r["hbm_gbs"], "frac_of_8TBs": r["frac_of_8TBs"],
+                             "frac": r["frac"], "read_probe_gbs": e["read_probe_gbs"]})
+        if rank == 0:
+            print(json.dumps({"metric": METRIC, "unit": UNIT, "sweep": rows, "steps": args.steps, "warmup": args.warmup,
+                              "peak": peaks}), flush=True)
+        return
 
     # ---- headline configuration ----
     t_wall0 = time.perf_counter()

@@ -53,6 +53,7 @@ extern "C" {
 #define IPPD_APPEND_CONTEXT 0
 #define IPPD_APPEND_QUESTION 1
 #define IPPD_APPEND_STEP 2
+#define IPPD_APPEND_SHARED 3
 
 /* keys of ippd_set_option */
 #define IPPD_OPT_KERNEL 1          /* 0 = auto, 1 = mma.sync path, 2 = tcgen05 path */
@@ -90,7 +91,9 @@ typedef struct {
   int32_t n_prompts, n_questions;
   int64_t n_header_tokens;
   int64_t n_branch_slots;      /* = branch_off[NQ] */
-  int64_t n_tiles;             /* context tiles + branch tiles of the whole cache, per layer and KV head */
+  int64_t n_tiles;             /* shared + context + branch tiles of the whole cache, per layer and KV head */
+  int32_t n_shared_tokens;     /* length of the instruction shared by all prompts (0 without one); the hdr_* arrays
+                                  start with its tokens (context id 0), hdr_begin[0] = n_shared_tokens */
 } ippd_tables_t;
 
 /*
@@ -110,6 +113,23 @@ typedef struct {
 int ippd_build_layout(const ippd_geometry_t* geom, int32_t n_prompts, const int32_t* ctx_len,
                       const int32_t* q_count, const int32_t* q_len, const int32_t* max_new,
                       ippd_layout_t** out);
+
+/*
+ * ippd_build_layout_shared -- ippd_build_layout for a batch whose prompts all start with the same
+ * instruction p of `shared_len` tokens (paper Sec. 4.1: stacked header [p, c_1, x_11, .., c_2, ..], p
+ * carries context id 0 and is attended by every token; Sec. 4.4: the instruction's K/V is kept once
+ * and reused by all stacked prompts of the batch).  Three levels of sharing: p by every question of
+ * the batch, context c_b by the questions of prompt b, a branch by its own question only.
+ *   pos_virt(token i of p)                     = i                      (cache tiles 0 .. ceil(shared_len/128)-1)
+ *   pos_virt(context token i of prompt b)      = shared_len + i
+ *   pos_virt(token j of question k, prompt b)  = shared_len + L_b + j
+ *   pos_virt(answer token fed at step s)       = shared_len + L_b + n_k + s
+ * p's K/V is appended once with ippd_append_kv(IPPD_APPEND_SHARED) and stored once; every row block's key
+ * sequence starts with p's tiles (tensor-core path only).  shared_len = 0 is ippd_build_layout.
+ */
+int ippd_build_layout_shared(const ippd_geometry_t* geom, int32_t shared_len, int32_t n_prompts,
+                             const int32_t* ctx_len, const int32_t* q_count, const int32_t* q_len,
+                             const int32_t* max_new, ippd_layout_t** out);
 
 /* Host views of the tables built above, for bit-exact comparison.  Host-only. */
 int ippd_layout_tables(const ippd_layout_t* layout, ippd_tables_t* out);
@@ -162,8 +182,9 @@ int ippd_step_descriptor_bytes(const ippd_layout_t* layout, const int32_t* activ
  * ippd_append_kv -- rotate raw keys to their virtual positions (RoPE, fp32 math on an
  * fp64-built table, result rounded to bf16) and store K and V into the cache
  * (paper Sec. 4.2, last paragraph: the token appended at each step carries its virtual position).
+ *   kind SHARED  : ids ignored; tokens = the shared instruction's tokens (ippd_build_layout_shared), position i.
  *   kind CONTEXT : ids[n_ids] = prompt ids (host); tokens = all context tokens of those
- *                  prompts, in id order; token i of prompt b gets position i.
+ *                  prompts, in id order; token i of prompt b gets position shared_len + i.
  *   kind QUESTION: ids[n_ids] = global question ids (host); tokens = their question
  *                  tokens in id order; token j gets position L_b + j, slot j of the branch.
  *   kind STEP    : ids ignored; one token per question of the last ippd_begin_step, in

@@ -76,14 +76,17 @@ def standalone_attend(k_raw: np.ndarray, v_raw: np.ndarray, q_raw: np.ndarray, t
 
 
 # --------------------------------------------------------------------------- integers
-def layout(ctx_len, q_count, q_len, max_new, branch_align: int, tile_tokens: int) -> dict:
-    """Integer tables of a batch of stacked prompts (one context per prompt).
+def layout(ctx_len, q_count, q_len, max_new, branch_align: int, tile_tokens: int, shared_len: int = 0) -> dict:
+    """Integer tables of a batch of stacked prompts (one context per prompt, an optional
+    instruction of `shared_len` tokens shared by all prompts).
 
-    Header of prompt b = its context tokens, then its questions' tokens in order.
-    Virtual positions: context token i -> i; token j of question k -> L_b + j; the
-    answer token fed at decode step s -> L_b + n_k + s.  Context ids are 1-based
-    per prompt (the instruction is folded into the context), question ids are
-    global and 1-based, 0 marks shared tokens.  Branch k owns slots
+    Header = the shared instruction's tokens (context id 0, question id 0), then per
+    prompt b its context tokens and its questions' tokens in order.  With P = shared_len,
+    virtual positions: instruction token i -> i; context token i -> P + i; token j of
+    question k -> P + L_b + j; the answer token fed at decode step s -> P + L_b + n_k + s
+    [Sec. 4.1].  Context ids are 1-based per prompt, question ids are global and
+    1-based, 0 marks shared tokens.  The instruction owns the first ceil(P / tile_tokens)
+    tiles.  Branch k owns slots
     [branch_off[k], branch_off[k+1]) with capacity n_k + max_new_k rounded up to
     `branch_align`; the answer token of step s lives at slot branch_off[k]+n_k+s.
     Context b owns tiles [ctx_tile_off[b], ctx_tile_off[b+1]) of `tile_tokens` tokens.
@@ -93,18 +96,21 @@ def layout(ctx_len, q_count, q_len, max_new, branch_align: int, tile_tokens: int
     for b in range(B):
         q_begin.append(q_begin[-1] + int(q_count[b]))
     NQ = q_begin[-1]
-    prompt_of, branch_off, hdr_begin = [], [0], [0]
+    P = int(shared_len)
+    prompt_of, branch_off, hdr_begin = [], [0], [P]
     pos, cid, qid = [], [], []
-    ctx_tile_off = [0]
+    for i in range(P):
+        pos.append(i); cid.append(0); qid.append(0)
+    ctx_tile_off = [(P + tile_tokens - 1) // tile_tokens]
     for b in range(B):
         L = int(ctx_len[b])
         ctx_tile_off.append(ctx_tile_off[-1] + (L + tile_tokens - 1) // tile_tokens)
         for i in range(L):
-            pos.append(i); cid.append(b + 1); qid.append(0)
+            pos.append(P + i); cid.append(b + 1); qid.append(0)
         for k in range(q_begin[b], q_begin[b + 1]):
             prompt_of.append(b)
             for j in range(int(q_len[k])):
-                pos.append(L + j); cid.append(b + 1); qid.append(k + 1)
+                pos.append(P + L + j); cid.append(b + 1); qid.append(k + 1)
             cap = int(q_len[k]) + int(max_new[k])
             cap = (cap + branch_align - 1) // branch_align * branch_align
             branch_off.append(branch_off[-1] + cap)
@@ -117,9 +123,9 @@ def layout(ctx_len, q_count, q_len, max_new, branch_align: int, tile_tokens: int
     }
 
 
-def step_position(ctx_len_b: int, q_len_k: int, s: int) -> int:
+def step_position(ctx_len_b: int, q_len_k: int, s: int, shared_len: int = 0) -> int:
     """Virtual position of the answer token fed at decode step s (the paper's t = s+1)."""
-    return ctx_len_b + q_len_k + s
+    return shared_len + ctx_len_b + q_len_k + s
 
 
 def stacked_sequence(p_len: int, ctx_lens, q_lens, n_answer, n_pad: int = 0):
@@ -194,9 +200,10 @@ def dense_attend(q_raw, k_raw, v_raw, pos, mask, theta: float) -> np.ndarray:
 def tuple_inputs(wl, b: int, k: int, s: int, layer: int, kv_head: int, ctx_cache: dict | None = None,
                  step_cache: dict | None = None):
     """Raw tensors of the standalone prompt of question k (global id) of prompt b at decode step s, one layer, one KV
-    head: (k_raw [T, D], v_raw [T, D], q_raw [G, D]) in fp64, T = L_b + n_k + s + 1.
+    head: (k_raw [T, D], v_raw [T, D], q_raw [G, D]) in fp64, T = P + L_b + n_k + s + 1.
 
-    The prompt is the context tokens, the question's tokens, then the answer tokens fed at steps 0..s (the last one is
+    The prompt is the instruction shared by the batch (P = wl.shared_len tokens, if the workload has one), the
+    context tokens, the question's tokens, then the answer tokens fed at steps 0..s (the last one is
     the token whose query is evaluated; Sec. 3, Sec. 4.2).  The G query heads [kv_head*G, (kv_head+1)*G) share KV head
     `kv_head`.  `wl` is any object with the raw-tensor accessors of a workload (ctx_kv, question_kv, step_kv, step_q,
     geom); the caches only avoid regenerating the same raw tensors.
@@ -215,6 +222,17 @@ def tuple_inputs(wl, b: int, k: int, s: int, layer: int, kv_head: int, ctx_cache
     kq, vq = wl.question_kv(k, layer)
     ks = [kc, kq[:, kv_head].double().numpy()]
     vs = [vc, vq[:, kv_head].double().numpy()]
+    if getattr(wl, "shared_len", 0) > 0:  # the triplet's prompt starts with the instruction p (Sec. 3: (p, c_j, x_jk))
+        skey = ("shared", layer, kv_head)
+        if ctx_cache is not None and skey in ctx_cache:
+            kp, vp = ctx_cache[skey]
+        else:
+            kp, vp = wl.shared_kv(layer)
+            kp, vp = kp[:, kv_head].double().numpy(), vp[:, kv_head].double().numpy()
+            if ctx_cache is not None:
+                ctx_cache[skey] = (kp, vp)
+        ks.insert(0, kp)
+        vs.insert(0, vp)
     for t in range(s + 1):
         if step_cache is None:
             ka, va = wl.step_kv(t, layer, [k])

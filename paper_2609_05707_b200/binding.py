@@ -21,10 +21,10 @@ OK, ERR_INVALID_ARG, ERR_OOM, ERR_CAPACITY, ERR_NOT_BOUND, ERR_CUDA, ERR_TIMEOUT
 BF16, F32 = 0, 1
 TILE_TOKENS = 128
 STATIC_SCRATCH_BYTES = 64 << 20
-APPEND_CONTEXT, APPEND_QUESTION, APPEND_STEP = 0, 1, 2
+APPEND_CONTEXT, APPEND_QUESTION, APPEND_STEP, APPEND_SHARED = 0, 1, 2, 3
 OPT_KERNEL, OPT_LAYERS_PER_CALL, OPT_TILES_PER_SPLIT, OPT_WAIT_LIMIT_US, OPT_PROFILE = 1, 2, 3, 4, 5
 
-EXPORTS = ["ippd_build_layout", "ippd_layout_tables", "ippd_cache_bytes", "ippd_bind_cache", "ippd_set_option",
+EXPORTS = ["ippd_build_layout", "ippd_build_layout_shared", "ippd_layout_tables", "ippd_cache_bytes", "ippd_bind_cache", "ippd_set_option",
            "ippd_begin_step", "ippd_step_descriptor_bytes", "ippd_append_kv", "ippd_workspace_bytes", "ippd_decode_attention", "ippd_decode_step", "ippd_decode_step_grouped", "ippd_decode_attention_static",
            "ippd_decode_step_host", "ippd_decode_step_host_async", "ippd_host_steps_wait", "ippd_step_stage_bytes", "ippd_export_mask", "ippd_poll_status", "ippd_profile_read", "ippd_read_probe", "ippd_host_time_read",
            "ippd_launch_count", "ippd_last_error", "ippd_destroy_layout"]
@@ -43,12 +43,13 @@ class Tables(C.Structure):
                 ("hdr_begin", C.POINTER(C.c_int64)), ("hdr_pos_virt", C.POINTER(C.c_int32)),
                 ("hdr_ctx_id", C.POINTER(C.c_int32)), ("hdr_qtn_id", C.POINTER(C.c_int32)),
                 ("n_prompts", C.c_int32), ("n_questions", C.c_int32), ("n_header_tokens", C.c_int64),
-                ("n_branch_slots", C.c_int64), ("n_tiles", C.c_int64)]
+                ("n_branch_slots", C.c_int64), ("n_tiles", C.c_int64), ("n_shared_tokens", C.c_int32)]
 
 
 _vp, _i32, _i64, _sz = C.c_void_p, C.c_int32, C.c_int64, C.c_size_t
 _pi32 = C.POINTER(C.c_int32)
 lib.ippd_build_layout.argtypes = [C.POINTER(Geometry), _i32, _pi32, _pi32, _pi32, _pi32, C.POINTER(_vp)]
+lib.ippd_build_layout_shared.argtypes = [C.POINTER(Geometry), _i32, _i32, _pi32, _pi32, _pi32, _pi32, C.POINTER(_vp)]
 lib.ippd_layout_tables.argtypes = [_vp, C.POINTER(Tables)]
 lib.ippd_cache_bytes.argtypes = [_vp, C.POINTER(_sz), C.POINTER(_sz)]
 lib.ippd_bind_cache.argtypes = [_vp, _vp, _sz, _vp]
@@ -110,14 +111,18 @@ def _dev(t) -> int:
 class Layout:
     """Owns one ippd_layout_t.  Methods mirror the C entry points one to one."""
 
-    def __init__(self, geom: Geometry, ctx_len, q_count, q_len, max_new):
+    def __init__(self, geom: Geometry, ctx_len, q_count, q_len, max_new, shared_len: int = 0):
         self.geom = geom
         self._h = _vp()
         c, qc, ql, mn = _i32arr(ctx_len), _i32arr(q_count), _i32arr(q_len), _i32arr(max_new)
         if len(c) != len(qc) or len(ql) != len(mn) or int(qc.sum()) != len(ql):
             raise ValueError("ragged arrays do not match")
-        _check(lib.ippd_build_layout(C.byref(geom), len(c), _p(c), _p(qc), _p(ql), _p(mn), C.byref(self._h)),
-               "ippd_build_layout")
+        if shared_len:
+            _check(lib.ippd_build_layout_shared(C.byref(geom), int(shared_len), len(c), _p(c), _p(qc), _p(ql), _p(mn),
+                                                C.byref(self._h)), "ippd_build_layout_shared")
+        else:
+            _check(lib.ippd_build_layout(C.byref(geom), len(c), _p(c), _p(qc), _p(ql), _p(mn), C.byref(self._h)),
+                   "ippd_build_layout")
         self._keep = None
 
     def close(self):
@@ -142,7 +147,7 @@ class Layout:
                 "hdr_begin": arr(t.hdr_begin, B + 1, np.int64), "hdr_pos_virt": arr(t.hdr_pos_virt, H, np.int32),
                 "hdr_ctx_id": arr(t.hdr_ctx_id, H, np.int32), "hdr_qtn_id": arr(t.hdr_qtn_id, H, np.int32),
                 "n_prompts": B, "n_questions": NQ, "n_header_tokens": H, "n_branch_slots": t.n_branch_slots,
-                "n_tiles": t.n_tiles}
+                "n_tiles": t.n_tiles, "n_shared_tokens": t.n_shared_tokens}
 
     def cache_bytes(self):
         b, a = _sz(), _sz()

@@ -111,7 +111,7 @@ static size_t ring_capacity(const IppdHostLayout& h) {
   size_t ctx_tiles_all_blocks = 0;  // whichever kernel path is selected later
   for (int b = 0; b < h.B; ++b) {
     const size_t blocks = (size_t)(h.q_count[b] + std::min(qpr_tc, qpr_mma) - 1) / std::min(qpr_tc, qpr_mma);
-    ctx_tiles_all_blocks += (size_t)(h.ctx_tile_off[b + 1] - h.ctx_tile_off[b]) * blocks;
+    ctx_tiles_all_blocks += (size_t)(h.n_shared_tiles + h.ctx_tile_off[b + 1] - h.ctx_tile_off[b]) * blocks;
   }
   const size_t nrb_any = std::max(nrb, (size_t)ceil_div_sz(h.NQ, 1));  // row blocks never outnumber questions
   const size_t units = ctx_tiles_all_blocks + branch_tiles + nrb_any + 2048;  // one unit per tile at worst
@@ -169,20 +169,27 @@ static IppdDev make_dev(const ippd_layout* L) {
   d.G = L->h.G;
   d.D = L->h.geom.head_dim;
   d.max_pos = L->h.max_pos;
+  d.shared_len = L->h.shared_len;
   return d;
+}
+
+extern "C" int ippd_build_layout_shared(const ippd_geometry_t* geom, int32_t shared_len, int32_t n_prompts,
+                                        const int32_t* ctx_len, const int32_t* q_count, const int32_t* q_len,
+                                        const int32_t* max_new, ippd_layout_t** out) {
+  if (!out) { ippd_set_error("ippd_build_layout: out is NULL"); return IPPD_ERR_INVALID_ARG; }
+  *out = nullptr;
+  ippd_layout* L = new (std::nothrow) ippd_layout();
+  if (!L) { ippd_set_error("ippd_build_layout: out of host memory"); return IPPD_ERR_OOM; }
+  int rc = ippd_host_build(geom, shared_len, n_prompts, ctx_len, q_count, q_len, max_new, &L->h);
+  if (rc != IPPD_OK) { delete L; return rc; }
+  *out = L;
+  return IPPD_OK;
 }
 
 extern "C" int ippd_build_layout(const ippd_geometry_t* geom, int32_t n_prompts, const int32_t* ctx_len,
                                  const int32_t* q_count, const int32_t* q_len, const int32_t* max_new,
                                  ippd_layout_t** out) {
-  if (!out) { ippd_set_error("ippd_build_layout: out is NULL"); return IPPD_ERR_INVALID_ARG; }
-  *out = nullptr;
-  ippd_layout* L = new (std::nothrow) ippd_layout();
-  if (!L) { ippd_set_error("ippd_build_layout: out of host memory"); return IPPD_ERR_OOM; }
-  int rc = ippd_host_build(geom, n_prompts, ctx_len, q_count, q_len, max_new, &L->h);
-  if (rc != IPPD_OK) { delete L; return rc; }
-  *out = L;
-  return IPPD_OK;
+  return ippd_build_layout_shared(geom, 0, n_prompts, ctx_len, q_count, q_len, max_new, out);
 }
 
 extern "C" int ippd_layout_tables(const ippd_layout_t* L, ippd_tables_t* t) {
@@ -203,6 +210,7 @@ extern "C" int ippd_layout_tables(const ippd_layout_t* L, ippd_tables_t* t) {
   t->n_header_tokens = (int64_t)h.hdr_pos.size();
   t->n_branch_slots = h.branch_off[h.NQ];
   t->n_tiles = h.n_tiles;
+  t->n_shared_tokens = h.shared_len;
   return IPPD_OK;
 }
 
@@ -397,7 +405,7 @@ extern "C" int ippd_begin_step(ippd_layout_t* L, const int32_t* active_q, const 
     int32_t* pos = reinterpret_cast<int32_t*>(blob.data() + off_pos);
     for (int a = 0; a < A; ++a) {
       const int k = P.act_q[a];
-      pos[a] = L->h.ctx_len[L->h.prompt_of[k]] + L->h.q_len[k] + P.act_s[a];
+      pos[a] = L->h.shared_len + L->h.ctx_len[L->h.prompt_of[k]] + L->h.q_len[k] + P.act_s[a];
     }
   }
   char* dev = nullptr;
@@ -474,6 +482,10 @@ extern "C" int ippd_append_kv(ippd_layout_t* L, int32_t layer_begin, int32_t lay
       int rc = ring_flush(L, stream);
       if (rc != IPPD_OK) return rc;
     }
+  } else if (kind == IPPD_APPEND_SHARED) {
+    a.n_tokens = h.shared_len;
+    int rc = ring_flush(L, stream);  // keeps the descriptor ring in stream order
+    if (rc != IPPD_OK) return rc;
   } else if (kind == IPPD_APPEND_CONTEXT || kind == IPPD_APPEND_QUESTION) {
     if (n_ids < 1 || !ids) { ippd_set_error("ippd_append_kv: ids missing"); return IPPD_ERR_INVALID_ARG; }
     std::vector<int32_t> blob((size_t)2 * n_ids + 4, 0);
@@ -995,8 +1007,8 @@ extern "C" int ippd_export_mask(ippd_layout_t* L, int32_t prompt, const int32_t*
   if (!L || !n_answer || !n_tokens) { ippd_set_error("ippd_export_mask: NULL argument"); return IPPD_ERR_INVALID_ARG; }
   const IppdHostLayout& h = L->h;
   if (prompt < 0 || prompt >= h.B) { ippd_set_error("ippd_export_mask: prompt out of range"); return IPPD_ERR_INVALID_ARG; }
-  std::vector<IppdMaskTok> toks;
-  for (int i = 0; i < h.ctx_len[prompt]; ++i) toks.push_back({0, -1, i, 0});
+  std::vector<IppdMaskTok> toks;  // shared instruction and context tokens: kind 0, idx = virtual position
+  for (int i = 0; i < h.shared_len + h.ctx_len[prompt]; ++i) toks.push_back({0, -1, i, 0});
   int k0 = h.q_begin[prompt], k1 = h.q_begin[prompt + 1];
   int max_t = 0;
   for (int k = k0; k < k1; ++k) {

@@ -112,9 +112,13 @@ ippd_append_kernel(IppdDev L, IppdStepDev S, IppdAppendArgs a, int layer_begin,
   if (a.kind == IPPD_APPEND_STEP) {
     int qid = a.inline_acts ? a.act_q[tok] : S.act_q[tok];
     int slot = L.q_len[qid] + (a.inline_acts ? a.act_s[tok] : S.act_s[tok]);
-    pos = L.ctx_len[L.prompt_of[qid]] + slot;
+    pos = L.shared_len + L.ctx_len[L.prompt_of[qid]] + slot;
     tile = L.branch_tile_off[qid] + slot / IPPD_TILE_TOKENS;
     u = slot % IPPD_TILE_TOKENS;
+  } else if (a.kind == IPPD_APPEND_SHARED) {
+    pos = tok;
+    tile = tok / IPPD_TILE_TOKENS;
+    u = tok % IPPD_TILE_TOKENS;
   } else {
     int lo = 0, hi = a.n_ids - 1;  // last id whose first token is <= tok
     while (lo < hi) {
@@ -123,10 +127,10 @@ ippd_append_kernel(IppdDev L, IppdStepDev S, IppdAppendArgs a, int layer_begin,
     }
     int id = a.ids[lo], i = tok - a.tok_begin[lo];
     if (a.kind == IPPD_APPEND_CONTEXT) {
-      pos = i;
+      pos = L.shared_len + i;
       tile = L.ctx_tile_off[id] + i / IPPD_TILE_TOKENS;
     } else {
-      pos = L.ctx_len[L.prompt_of[id]] + i;
+      pos = L.shared_len + L.ctx_len[L.prompt_of[id]] + i;
       tile = L.branch_tile_off[id] + i / IPPD_TILE_TOKENS;
     }
     u = i % IPPD_TILE_TOKENS;

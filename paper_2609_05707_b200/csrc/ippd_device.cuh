@@ -23,6 +23,7 @@ struct IppdDev {
   long long n_tiles;
   long long wait_limit_ns;
   int n_layers, Hq, Hkv, G, D, max_pos;
+  int shared_len;  // tokens of the instruction shared by all prompts (positions 0 .. shared_len-1, tiles from 0)
 };
 
 // Per-step arrays (device pointers into the step blob).

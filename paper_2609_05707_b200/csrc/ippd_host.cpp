@@ -23,13 +23,14 @@ static int questions_per_block(const IppdHostLayout& L) {
 
 static inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
 
-int ippd_host_build(const ippd_geometry_t* g, int32_t B, const int32_t* ctx_len, const int32_t* q_count,
-                    const int32_t* q_len, const int32_t* max_new, IppdHostLayout* L) {
+int ippd_host_build(const ippd_geometry_t* g, int32_t shared_len, int32_t B, const int32_t* ctx_len,
+                    const int32_t* q_count, const int32_t* q_len, const int32_t* max_new, IppdHostLayout* L) {
   if (!g || !ctx_len || !q_count || !q_len || !max_new || !L) {
     ippd_set_error("ippd_build_layout: NULL argument");
     return IPPD_ERR_INVALID_ARG;
   }
   if (B < 1) { ippd_set_error("ippd_build_layout: n_prompts must be >= 1"); return IPPD_ERR_INVALID_ARG; }
+  if (shared_len < 0) { ippd_set_error("ippd_build_layout: shared_len < 0"); return IPPD_ERR_INVALID_ARG; }
   if (g->n_layers < 1 || g->n_kv_heads < 1 || g->n_q_heads < 1 || g->n_q_heads % g->n_kv_heads != 0) {
     ippd_set_error("ippd_build_layout: bad head counts / layers");
     return IPPD_ERR_INVALID_ARG;
@@ -54,6 +55,8 @@ int ippd_host_build(const ippd_geometry_t* g, int32_t B, const int32_t* ctx_len,
   }
   try {
     L->geom = *g;
+    L->shared_len = shared_len;
+    L->n_shared_tiles = (int32_t)ceil_div(shared_len, IPPD_TILE_TOKENS);
     L->B = B;
     L->G = G;
     L->ctx_len.assign(ctx_len, ctx_len + B);
@@ -74,8 +77,9 @@ int ippd_host_build(const ippd_geometry_t* g, int32_t B, const int32_t* ctx_len,
     L->branch_off.assign(nq + 1, 0);
     L->branch_tile_off.assign(nq + 1, 0);
     L->hdr_begin.assign(B + 1, 0);
-    L->ctx_tile_off.assign(B + 1, 0);
-    int64_t max_pos = 0, hdr = 0;
+    L->ctx_tile_off.assign(B + 1, L->n_shared_tiles);  // the shared instruction owns the first tiles of the cache
+    int64_t max_pos = 0, hdr = shared_len;
+    L->hdr_begin[0] = shared_len;
     for (int b = 0; b < B; ++b) {
       L->ctx_tile_off[b + 1] = L->ctx_tile_off[b] + (int32_t)ceil_div(ctx_len[b], IPPD_TILE_TOKENS);
       hdr += ctx_len[b];
@@ -84,7 +88,7 @@ int ippd_host_build(const ippd_geometry_t* g, int32_t B, const int32_t* ctx_len,
           ippd_set_error("ippd_build_layout: q_len and max_new must be >= 1");
           return IPPD_ERR_INVALID_ARG;
         }
-        int64_t last = (int64_t)ctx_len[b] + q_len[k] + max_new[k];
+        int64_t last = (int64_t)shared_len + ctx_len[b] + q_len[k] + max_new[k];
         if (last >= INT32_MAX) { ippd_set_error("ippd_build_layout: position overflows int32"); return IPPD_ERR_INVALID_ARG; }
         max_pos = std::max(max_pos, last - 1);
         L->prompt_of[k] = b;
@@ -101,14 +105,16 @@ int ippd_host_build(const ippd_geometry_t* g, int32_t B, const int32_t* ctx_len,
     L->n_tiles = n_tiles;
     for (int64_t k = 0; k <= nq; ++k)
       L->branch_tile_off[k] = (int32_t)(L->n_ctx_tiles + L->branch_off[k] / IPPD_TILE_TOKENS);
-    // stacked-header metadata: context tokens, then the question blocks
+    // stacked-header metadata: the shared instruction (context id 0: everybody's), then per prompt its context
+    // tokens and question blocks
     L->hdr_pos.resize(hdr); L->hdr_ctx.resize(hdr); L->hdr_qtn.resize(hdr);
     int64_t h = 0;
+    for (int i = 0; i < shared_len; ++i, ++h) { L->hdr_pos[h] = i; L->hdr_ctx[h] = 0; L->hdr_qtn[h] = 0; }
     for (int b = 0; b < B; ++b) {
-      for (int i = 0; i < ctx_len[b]; ++i, ++h) { L->hdr_pos[h] = i; L->hdr_ctx[h] = b + 1; L->hdr_qtn[h] = 0; }
+      for (int i = 0; i < ctx_len[b]; ++i, ++h) { L->hdr_pos[h] = shared_len + i; L->hdr_ctx[h] = b + 1; L->hdr_qtn[h] = 0; }
       for (int k = L->q_begin[b]; k < L->q_begin[b + 1]; ++k)
         for (int j = 0; j < q_len[k]; ++j, ++h) {
-          L->hdr_pos[h] = ctx_len[b] + j; L->hdr_ctx[h] = b + 1; L->hdr_qtn[h] = k + 1;
+          L->hdr_pos[h] = shared_len + ctx_len[b] + j; L->hdr_ctx[h] = b + 1; L->hdr_qtn[h] = k + 1;
         }
     }
   } catch (const std::bad_alloc&) {
@@ -132,7 +138,7 @@ int64_t ippd_host_max_units(const IppdHostLayout& L, int32_t layer_count) {
     int64_t tiles = 0;
     int qpr = questions_per_block(L);
     for (int b = 0; b < L.B; ++b) {
-      tiles += ceil_div(L.q_count[b], qpr) * (L.ctx_tile_off[b + 1] - L.ctx_tile_off[b]);
+      tiles += ceil_div(L.q_count[b], qpr) * (L.n_shared_tiles + L.ctx_tile_off[b + 1] - L.ctx_tile_off[b]);
       tiles += L.branch_tile_off[L.q_begin[b + 1]] - L.branch_tile_off[L.q_begin[b]];
     }
     return nrb + ceil_div(tiles, L.opt_tiles_per_split);
@@ -156,6 +162,10 @@ int ippd_host_plan_step(const IppdHostLayout& L, const int32_t* active_q, const 
   plan->tc_tiles.clear();
   plan->tc_pieces.clear();
   const bool tc_path = L.kernel_path() == 2;
+  if (!tc_path && L.shared_len > 0) {
+    ippd_set_error("ippd_begin_step: a shared instruction needs the tensor-core path (IPPD_OPT_KERNEL 0 or 2)");
+    return IPPD_ERR_INVALID_ARG;
+  }
   int64_t total = 0;
   int i = 0;
   int32_t prev = -1;
@@ -172,7 +182,8 @@ int ippd_host_plan_step(const IppdHostLayout& L, const int32_t* active_q, const 
       prev = k;
       ++j;
     }
-    int nct = L.ctx_tile_off[b + 1] - L.ctx_tile_off[b];
+    const int nct_own = L.ctx_tile_off[b + 1] - L.ctx_tile_off[b];
+    const int nct = L.n_shared_tiles + nct_own;  // every query row sees the shared instruction, then its own context
     for (int a0 = i; a0 < j; a0 += qpr) {
       IppdRowBlock rb;
       memset(&rb, 0, sizeof(rb));
@@ -182,7 +193,11 @@ int ippd_host_plan_step(const IppdHostLayout& L, const int32_t* active_q, const 
       rb.n_ctx_tiles = nct;
       int64_t tiles = nct;
       if (tc_path) {
-        for (int t = 0; t < nct; ++t) {
+        for (int t = 0; t < L.n_shared_tiles; ++t) {
+          IppdTcTile ti = {t, std::min(IPPD_TILE_TOKENS, L.shared_len - t * IPPD_TILE_TOKENS), 0, 0};
+          plan->tc_tiles.push_back(ti);
+        }
+        for (int t = 0; t < nct_own; ++t) {
           IppdTcTile ti = {L.ctx_tile_off[b] + t, std::min(IPPD_TILE_TOKENS, L.ctx_len[b] - t * IPPD_TILE_TOKENS), 0, 0};
           plan->tc_tiles.push_back(ti);
         }

@@ -76,7 +76,8 @@ struct IppdHostLayout {
   std::vector<int64_t> branch_off, hdr_begin;
   std::vector<int32_t> branch_tile_off;  // [NQ+1] global tile index (context tiles come first)
   std::vector<int32_t> hdr_pos, hdr_ctx, hdr_qtn;
-  int64_t n_ctx_tiles = 0, n_tiles = 0;
+  int64_t n_ctx_tiles = 0, n_tiles = 0;  // n_ctx_tiles counts the shared instruction's tiles too
+  int32_t shared_len = 0, n_shared_tiles = 0;  // instruction shared by every prompt of the batch: tiles [0, n_shared_tiles)
   int32_t max_pos = 0;
   // options
   int32_t opt_kernel = 0, opt_layers_per_call = 0, opt_tiles_per_split = 0;
@@ -91,7 +92,7 @@ struct IppdHostLayout {
 };
 
 void ippd_set_error(const std::string& msg);
-int ippd_host_build(const ippd_geometry_t* geom, int32_t n_prompts, const int32_t* ctx_len,
+int ippd_host_build(const ippd_geometry_t* geom, int32_t shared_len, int32_t n_prompts, const int32_t* ctx_len,
                     const int32_t* q_count, const int32_t* q_len, const int32_t* max_new,
                     IppdHostLayout* out);
 // Builds the work list of one step.  Returns IPPD_OK or an error code.

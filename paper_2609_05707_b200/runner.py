@@ -29,7 +29,7 @@ class Runner:
         g = wl.geom
         self.geom = B.make_geometry(g.n_layers, g.n_q_heads, g.n_kv_heads, g.head_dim, g.rope_theta,
                                     branch_align, out_dtype)
-        self.layout = B.Layout(self.geom, wl.ctx_len, wl.q_count, wl.q_len, wl.max_new)
+        self.layout = B.Layout(self.geom, wl.ctx_len, wl.q_count, wl.q_len, wl.max_new, shared_len=wl.shared_len)
         if kernel:
             self.layout.set_option(B.OPT_KERNEL, kernel)
         if layers_per_call:
@@ -61,6 +61,9 @@ class Runner:
         prompts = list(range(wl.n_prompts)) if prompts is None else list(prompts)
         qids = [k for b in prompts for k in range(int(wl.q_begin[b]), int(wl.q_begin[b + 1]))]
         for layer in range(g.n_layers):
+            if wl.shared_len > 0:
+                k, v = wl.shared_kv(layer, self.device)
+                self.layout.append_kv(layer, 1, B.APPEND_SHARED, None, k, v, self.stream)
             for b in prompts:
                 if wl.ctx_len[b] == 0:
                     continue

@@ -79,7 +79,7 @@ def normal_table(device="cpu") -> torch.Tensor:
 
 
 # tensor stream kinds
-K_CTX, V_CTX, K_QST, V_QST, Q_STEP, K_STEP, V_STEP = 1, 2, 3, 4, 5, 6, 7
+K_CTX, V_CTX, K_QST, V_QST, Q_STEP, K_STEP, V_STEP, K_SHR, V_SHR = 1, 2, 3, 4, 5, 6, 7, 8, 9
 
 
 def stream_id(kind: int, index: int) -> int:
@@ -136,6 +136,7 @@ class Workload:
     stop: np.ndarray         # [NQ] int32: question k is active at steps 0..stop[k]-1
     max_new: np.ndarray      # [NQ] int32: branch capacity in answer tokens
     n_steps: int
+    shared_len: int = 0      # tokens of an instruction shared by every prompt of the batch (0 = none)
     q_begin: np.ndarray = field(init=False)
     prompt_of: np.ndarray = field(init=False)
 
@@ -165,7 +166,8 @@ class Workload:
         act = self.active(s)
         kvb = g.kv_bytes_per_token
         prompts = np.unique(self.prompt_of[act])
-        ctx = int(self.ctx_len[prompts].astype(np.int64).sum()) * kvb
+        # the shared instruction is read once for the whole batch, a context once per prompt with an active question
+        ctx = (int(self.ctx_len[prompts].astype(np.int64).sum()) + (self.shared_len if len(act) else 0)) * kvb
         br = int((self.q_len[act].astype(np.int64) + s + 1).sum()) * kvb
         qo = len(act) * g.n_q_heads * g.head_dim * 2 * 2
         return {"context": ctx * g.n_layers, "branch": br * g.n_layers, "q_out": qo * g.n_layers,
@@ -174,7 +176,7 @@ class Workload:
     def step_flops(self, s: int) -> int:
         g = self.geom
         act = self.active(s)
-        keys = (self.ctx_len[self.prompt_of[act]].astype(np.int64) + self.q_len[act] + s + 1).sum()
+        keys = (self.shared_len + self.ctx_len[self.prompt_of[act]].astype(np.int64) + self.q_len[act] + s + 1).sum()
         return int(4 * g.head_dim * g.n_q_heads * keys) * g.n_layers
 
     # ---- raw tensors (bf16), generated on the requested device ----
@@ -191,6 +193,13 @@ class Workload:
         shape = (t1 - t0, g.n_kv_heads, g.head_dim)
         row0 = layer * L + t0
         return (self._gen(K_CTX, b, shape, row0, device), self._gen(V_CTX, b, shape, row0, device))
+
+    def shared_kv(self, layer: int, device="cpu"):
+        """Raw K and V of the shared instruction's tokens at one layer: [shared_len, Hkv, D]."""
+        g = self.geom
+        shape = (self.shared_len, g.n_kv_heads, g.head_dim)
+        row0 = layer * self.shared_len
+        return (self._gen(K_SHR, 0, shape, row0, device), self._gen(V_SHR, 0, shape, row0, device))
 
     def question_kv(self, k: int, layer: int, device="cpu"):
         """Raw K and V of question k's own tokens at one layer: [n_k, Hkv, D]."""
@@ -235,6 +244,8 @@ def make_workload(name: str, n_layers: Optional[int] = None) -> Workload:
     layers kept are unchanged because the layer is the slowest index only within
     a layer's own slice for per-token tensors -- see ctx_kv/question_kv).
     """
+    if name.startswith("SWEEP-"):
+        return _sweep_workload(name, n_layers)
     if name.startswith("S"):
         return _shape_workload(name, n_layers)
     c = int(name[1:])
@@ -279,13 +290,19 @@ def _shape_workload(name: str, n_layers: Optional[int] = None) -> Workload:
 
     S1  long contexts, many questions, short answers: L ~ U{2600..4400}, Q ~ U{22..38}, n ~ U{8..16}, stop ~ U{6..40}
     S2  short contexts, few questions:                L ~ U{170..280},   Q ~ U{6..12},  n ~ U{9..17}, stop ~ U{4..30}
+    S3  a long instruction shared by the whole batch (few-shot examples, kept once): P = 2754 tokens, twelve prompts
+        (three stacked prompts of four contexts in the paper's terms) with L ~ U{550..920}, Q ~ U{22..38},
+        n ~ U{8..16}, stop ~ U{1..11}
     """
     c = int(name[1:])
     seed = _BASE_SEED + 100 + c
     ri = lambda tag, i, lo, hi: _randint(seed, tag, i, lo, hi)
-    B = 6
+    B, shared = 6, 0
     if c == 1:
         Lr, Qr, nr, sr = (2600, 4400), (22, 38), (8, 16), (6, 40)
+    elif c == 3:
+        B, shared = 12, 2754
+        Lr, Qr, nr, sr = (550, 920), (22, 38), (8, 16), (1, 11)
     elif c == 2:
         Lr, Qr, nr, sr = (170, 280), (6, 12), (9, 17), (4, 30)
     else:
@@ -299,12 +316,33 @@ def _shape_workload(name: str, n_layers: Optional[int] = None) -> Workload:
     q_len = np.array([ri(3, k, *nr) for k in range(NQ)], dtype=np.int32)
     stop = np.array([ri(4, k, *sr) for k in range(NQ)], dtype=np.int32)
     return Workload(name, geom, seed, np.array(ctx, dtype=np.int32), np.array(qc, dtype=np.int32), q_len, stop,
-                    stop.copy(), int(stop.max()))
+                    stop.copy(), int(stop.max()), shared)
+
+
+SWEEP_CONTEXTS = (2048, 4096, 8192, 16384)
+SWEEP_QUESTIONS = (1, 2, 4, 8, 16, 32)
+
+
+def _sweep_workload(name: str, n_layers: Optional[int] = None) -> Workload:
+    """The axes of the paper's ablations (App. C: questions per context 1..32, context length 1x..8x) as named
+    workloads "SWEEP-L<context>-Q<questions>": one prompt with a context of L tokens and Q questions of 32 tokens each,
+    16 decode steps without stop steps, Llama-3-8B geometry."""
+    parts = name.split("-")
+    L, Q = int(parts[1][1:]), int(parts[2][1:])
+    assert parts[0] == "SWEEP" and 1 <= L <= (1 << 20) and 1 <= Q <= 4096, name
+    geom = LLAMA3_8B
+    if n_layers is not None:
+        geom = Geometry(n_layers, geom.n_q_heads, geom.n_kv_heads, geom.head_dim, geom.rope_theta)
+    seed = _BASE_SEED + 1000 + 64 * (L // 1024) + Q
+    stop = np.full(Q, 16, dtype=np.int32)
+    return Workload(name, geom, seed, np.array([L], dtype=np.int32), np.array([Q], dtype=np.int32),
+                    np.full(Q, 32, dtype=np.int32), stop, stop.copy(), 16)
 
 
 def custom_workload(name: str, geom: Geometry, seed: int, ctx_len: List[int], q_count: List[int],
-                    q_len: List[int], stop: List[int], max_new: Optional[List[int]] = None) -> Workload:
+                    q_len: List[int], stop: List[int], max_new: Optional[List[int]] = None,
+                    shared_len: int = 0) -> Workload:
     stop_a = np.array(stop, dtype=np.int32)
     mn = stop_a.copy() if max_new is None else np.array(max_new, dtype=np.int32)
     return Workload(name, geom, seed, np.array(ctx_len, dtype=np.int32), np.array(q_count, dtype=np.int32),
-                    np.array(q_len, dtype=np.int32), stop_a, mn, int(stop_a.max()))
+                    np.array(q_len, dtype=np.int32), stop_a, mn, int(stop_a.max()), shared_len)

@@ -35,9 +35,11 @@ def test_layout_tables_bit_exact_vs_oracle(seed):
     ql = r.integers(1, 70, nq)
     mn = r.integers(1, 300, nq)
     align = int(r.choice([128, 256]))
-    lay = B.Layout(B.make_geometry(2, 8, 2, 64, 1e4, branch_align=align), ctx, qc, ql, mn)
+    shared = int([0, 1, 127, 128, 300, 0][seed])  # an instruction shared by all prompts
+    lay = B.Layout(B.make_geometry(2, 8, 2, 64, 1e4, branch_align=align), ctx, qc, ql, mn, shared_len=shared)
     got = lay.layout_tables()
-    want = orc.layout(ctx, qc, ql, mn, align, B.TILE_TOKENS)
+    want = orc.layout(ctx, qc, ql, mn, align, B.TILE_TOKENS, shared_len=shared)
+    assert got["n_shared_tokens"] == shared and got["n_header_tokens"] == len(want["hdr_pos_virt"])
     for key in ["q_begin", "prompt_of", "branch_off", "ctx_tile_off", "hdr_begin", "hdr_pos_virt", "hdr_ctx_id",
                 "hdr_qtn_id"]:
         np.testing.assert_array_equal(got[key], want[key], err_msg=key)

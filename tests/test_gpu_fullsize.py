@@ -131,3 +131,10 @@ def test_s2_full_size_sampled():
     lh = _layer_heads(wl, [(7, 5), (19, 2), (26, 6), (3, 3), (29, 1), (14, 7), (22, 0), (10, 4)])
     n = run_and_sample("S2", {s: lh for s in _steps(wl, [3])}, per_prompt=12)
     assert n >= MIN_TUPLES, n
+
+
+@pytest.mark.parametrize("name", ["SWEEP-L2048-Q1", "SWEEP-L2048-Q32", "SWEEP-L16384-Q1", "SWEEP-L16384-Q32"])
+def test_sweep_corners_sampled(name):
+    # the four corners of the questions-per-context x context-length sweep (the axes of the paper's ablations)
+    wl = W.make_workload(name)
+    run_and_sample(name, {0: [(0, 0), (31, 7)], 15: [(0, 0), (16, 3), (31, 7)]}, per_prompt=8)

@@ -306,3 +306,81 @@ def test_attend_tuple_equals_the_dense_mask_formulation():
                             np.testing.assert_allclose(got[j], dense[(k, kv_head * G + j)], atol=1e-12, rtol=0)
                             checked += 1
         assert checked == int(wl.stop.sum()) * hq
+
+
+def _dense_rows_of_batch_step(wl, s, layer):
+    """The whole batch as ONE stacked sequence [p, c_1, x_11, .., c_2, x_21, ..] (Sec. 4.1): the shared instruction p
+    with context id 0, every prompt of the batch as one context of the stacked prompt, then the answer tokens.  Returns
+    the dense-mask attention rows of the answer tokens fed at step s, per query head, assembled from the raw accessors
+    without attend_tuple."""
+    g = wl.geom
+    G = g.n_q_heads // g.n_kv_heads
+    P = wl.shared_len
+    B = wl.n_prompts
+    q_lens = [[int(wl.q_len[k]) for k in range(int(wl.q_begin[b]), int(wl.q_begin[b + 1]))] for b in range(B)]
+    n_answer = [[min(int(wl.stop[k]), s + 1) for k in range(int(wl.q_begin[b]), int(wl.q_begin[b + 1]))]
+                for b in range(B)]
+    pos, ctx, qtn, tag = orc.stacked_sequence(P, [int(v) for v in wl.ctx_len], q_lens, n_answer)
+    mask = orc.dense_mask(pos, ctx, qtn)
+    n = len(pos)
+    K = np.zeros((n, g.n_kv_heads, g.head_dim))
+    V = np.zeros_like(K)
+    Q = np.zeros((n, g.n_q_heads, g.head_dim))
+    kp, vp = wl.shared_kv(layer) if P else (None, None)
+    rows = {}
+    for i, (kind, j, kk, idx) in enumerate(tag):
+        k = int(wl.q_begin[j]) + kk
+        if kind == "p":
+            K[i], V[i] = kp[idx].double().numpy(), vp[idx].double().numpy()
+        elif kind == "c":
+            kc, vc = wl.ctx_kv(j, layer, t0=idx, t1=idx + 1)
+            K[i], V[i] = kc[0].double().numpy(), vc[0].double().numpy()
+        elif kind == "x":
+            kq, vq = wl.question_kv(k, layer)
+            K[i], V[i] = kq[idx].double().numpy(), vq[idx].double().numpy()
+        else:
+            ka, va = wl.step_kv(idx, layer, [k])
+            K[i], V[i] = ka[0].double().numpy(), va[0].double().numpy()
+            if idx == s:
+                Q[i] = wl.step_q(s, layer, [k])[0].double().numpy()
+                rows[k] = i
+    K_rep, V_rep = np.repeat(K, G, axis=1), np.repeat(V, G, axis=1)
+    out = {}
+    for h in range(g.n_q_heads):
+        o = orc.dense_attend(Q[:, h], K_rep[:, h], V_rep[:, h], pos, mask, g.rope_theta)
+        for k, i in rows.items():
+            out[(k, h)] = o[i]
+    return out
+
+
+@pytest.mark.parametrize("shared_len", [0, 6])
+def test_attend_tuple_equals_one_stacked_prompt_with_several_contexts(shared_len):
+    # Sec. 4.1 / 4.4: several contexts stacked in one prompt behind a shared instruction p (context id 0, attended by
+    # everybody; M_ctx keeps the contexts apart).  The standalone prompt of a triplet is (p, c_j, x_jk, answers); its
+    # output must equal the dense-mask row over the whole stacked batch.  A wrong position offset for p, a context
+    # leaking into another context's questions, or p missing from the standalone prompt each break the agreement.
+    from paper_2609_05707_b200 import workloads as W
+    wl = W.custom_workload("pin3", W.Geometry(1, 4, 2, 16, 1e4), 78, [5, 0, 7], [2, 1, 2], [2, 3, 1, 2, 4],
+                           [3, 2, 1, 3, 2], shared_len=shared_len)
+    checked = 0
+    for s in range(wl.n_steps):
+        dense = _dense_rows_of_batch_step(wl, s, 0)
+        act = [int(k) for k in wl.active(s)]
+        assert sorted({k for k, _ in dense}) == act
+        for k in act:
+            for kv_head in range(2):
+                got = orc.attend_tuple(wl, int(wl.prompt_of[k]), k, s, 0, kv_head)
+                for j in range(2):
+                    np.testing.assert_allclose(got[j], dense[(k, kv_head * 2 + j)], atol=1e-12, rtol=0)
+                    checked += 1
+    assert checked == int(wl.stop.sum()) * 4
+
+
+def test_layout_with_a_shared_instruction():
+    # closed forms of Sec. 4.1 with an instruction of P tokens: p -> [0, P), c_b -> [P, P + L_b), x_k -> from P + L_b
+    lay = orc.layout([3, 2], [1, 2], [2, 1, 3], [4, 4, 4], 128, 128, shared_len=5)
+    assert lay["hdr_pos_virt"].tolist() == [0, 1, 2, 3, 4, 5, 6, 7, 8, 9, 5, 6, 7, 7, 8, 9]
+    assert lay["hdr_ctx_id"].tolist() == [0] * 5 + [1] * 5 + [2] * 6
+    assert lay["hdr_qtn_id"].tolist() == [0] * 5 + [0, 0, 0, 1, 1] + [0, 0, 2, 3, 3, 3]
+    assert lay["hdr_begin"].tolist() == [5, 10, 16] and lay["ctx_tile_off"].tolist() == [1, 2, 3]
+    assert orc.step_position(3, 2, 4, shared_len=5) == 14

@@ -56,3 +56,18 @@ def test_config_shapes_follow_the_recipe():
     assert torch.equal(a, b)
     sb = c2.step_bytes(0)
     assert sb["context"] == 2048 * 4096 * 32 and sb["branch"] == int((c2.q_len + 1).sum()) * 4096 * 32
+
+
+def test_sweep_and_shared_workloads_follow_their_recipes():
+    wl = W.make_workload("SWEEP-L8192-Q4")
+    assert wl.ctx_len.tolist() == [8192] and wl.q_count.tolist() == [4] and wl.q_len.tolist() == [32] * 4
+    assert wl.n_steps == 16 and (wl.stop == 16).all() and wl.geom.n_layers == 32
+    assert W.make_workload("SWEEP-L2048-Q32", n_layers=2).geom.n_layers == 2
+    s3 = W.make_workload("S3")
+    assert s3.shared_len == 2754 and s3.n_prompts == 12
+    assert (s3.ctx_len >= 550).all() and (s3.ctx_len <= 920).all() and (s3.stop >= 1).all() and (s3.stop <= 11).all()
+    k, v = s3.shared_kv(3)
+    assert k.shape == (2754, 8, 128) and not torch.equal(k, v)
+    # the instruction is counted once per step in the algorithmic bytes, every context once
+    b = s3.step_bytes(0)
+    assert b["context"] == (2754 + int(s3.ctx_len.sum())) * s3.geom.kv_bytes_per_token * 32
