@@ -23,6 +23,9 @@ What is defined here (paper sections in brackets):
   tiny inputs to show that it agrees with `standalone_attend` (the paper's
   equivalence claim) and that the structural attended set equals the predicates.
 
+* `standalone_prefill`, `prefill_tuple` -- the prefill of the stacked header: every header row
+  equals the row of its own standalone causal prompt [Sec. 4, Sec. 4.2].  Pinned by: the library
+  SDPA with is_causal, and the dense formulation (header rows under the dense mask).
 * `tuple_inputs`, `attend_tuple` -- assemble the standalone prompt of one (prompt,
   question, step, layer, KV head) from a workload's raw accessors and evaluate it.
   Pinned by: the dense formulation over a stacked sequence assembled independently
@@ -73,6 +76,33 @@ def standalone_attend(k_raw: np.ndarray, v_raw: np.ndarray, q_raw: np.ndarray, t
     p = np.exp(z)
     p = p / p.sum(axis=-1, keepdims=True)
     return p @ v
+
+
+def standalone_prefill(k_raw: np.ndarray, v_raw: np.ndarray, q_raw: np.ndarray, theta: float) -> np.ndarray:
+    """Causal self-attention of ONE standalone prompt, every row (the prefill of a triplet prompted alone).
+
+    k_raw, v_raw: [T, D] raw keys / values of the prompt's T tokens; q_raw: [T, H, D] raw queries of the same tokens
+    for the H query heads that share this KV head.  Ordinary positions 0..T-1; row i sees keys 0..i.  Returns
+    [T, H, D] fp64.  [Sec. 4: the stacked header is prefilled once; Sec. 4.2: every token of the stacked prompt follows
+    the computation of its own standalone prompt.]
+    """
+    k_raw = np.asarray(k_raw, dtype=np.float64)
+    v = np.asarray(v_raw, dtype=np.float64)
+    q_raw = np.asarray(q_raw, dtype=np.float64)
+    T, D = k_raw.shape
+    pos = np.arange(T)
+    k = rope(k_raw, pos, theta)
+    out = np.empty_like(q_raw)
+    causal = np.tril(np.ones((T, T), dtype=bool))
+    for h in range(q_raw.shape[1]):
+        q = rope(q_raw[:, h], pos, theta)
+        z = (q @ k.T) / np.sqrt(D)
+        z = np.where(causal, z, -np.inf)
+        z = z - z.max(axis=-1, keepdims=True)
+        p = np.exp(z)
+        p = p / p.sum(axis=-1, keepdims=True)
+        out[:, h] = p @ v
+    return out
 
 
 # --------------------------------------------------------------------------- integers
@@ -254,3 +284,28 @@ def attend_tuple(wl, b: int, k: int, s: int, layer: int, kv_head: int, ctx_cache
     dense-mask formulation assembled independently in the tests (the equivalence of Sec. 4.2)."""
     k_raw, v_raw, q_raw = tuple_inputs(wl, b, k, s, layer, kv_head, ctx_cache, step_cache)
     return standalone_attend(k_raw, v_raw, q_raw, wl.geom.rope_theta)
+
+
+def prefill_tuple(wl, b: int, k: int | None, layer: int, kv_head: int) -> np.ndarray:
+    """Oracle prefill outputs of the header rows of one standalone prompt, one layer, all query heads of one KV head.
+
+    k = a global question id: the prompt is (instruction p, context c_b, question x_k); returns the rows of the
+    question's tokens, [n_k, G, D].  k = None: the prompt is (p, c_b) alone; returns the rows of p and c_b,
+    [P + L_b, G, D] (a context row does not depend on the questions behind it).  Uses the workload's header query
+    accessors (shared_q, ctx_q, question_q) next to the key/value accessors.
+    """
+    g = wl.geom
+    G = g.n_q_heads // g.n_kv_heads
+    hs = slice(kv_head * G, (kv_head + 1) * G)
+    ks, vs, qs = [], [], []
+    if getattr(wl, "shared_len", 0) > 0:
+        kp, vp = wl.shared_kv(layer)
+        ks.append(kp[:, kv_head]); vs.append(vp[:, kv_head]); qs.append(wl.shared_q(layer)[:, hs])
+    kc, vc = wl.ctx_kv(b, layer)
+    ks.append(kc[:, kv_head]); vs.append(vc[:, kv_head]); qs.append(wl.ctx_q(b, layer)[:, hs])
+    if k is not None:
+        kq, vq = wl.question_kv(k, layer)
+        ks.append(kq[:, kv_head]); vs.append(vq[:, kv_head]); qs.append(wl.question_q(k, layer)[:, hs])
+    cat = lambda ts: np.concatenate([t.double().numpy() for t in ts])
+    out = standalone_prefill(cat(ks), cat(vs), cat(qs), g.rope_theta)
+    return out if k is None else out[-int(wl.q_len[k]):]

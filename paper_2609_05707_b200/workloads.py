@@ -79,7 +79,7 @@ def normal_table(device="cpu") -> torch.Tensor:
 
 
 # tensor stream kinds
-K_CTX, V_CTX, K_QST, V_QST, Q_STEP, K_STEP, V_STEP, K_SHR, V_SHR = 1, 2, 3, 4, 5, 6, 7, 8, 9
+K_CTX, V_CTX, K_QST, V_QST, Q_STEP, K_STEP, V_STEP, K_SHR, V_SHR, Q_CTX, Q_QST, Q_SHR = 1, 2, 3, 4, 5, 6, 7, 8, 9, 10, 11, 12
 
 
 def stream_id(kind: int, index: int) -> int:
@@ -207,6 +207,24 @@ class Workload:
         n = int(self.q_len[k])
         shape = (n, g.n_kv_heads, g.head_dim)
         return (self._gen(K_QST, k, shape, layer * n, device), self._gen(V_QST, k, shape, layer * n, device))
+
+    # ---- raw queries of the header tokens (prefill) ----
+    def shared_q(self, layer: int, device="cpu") -> torch.Tensor:
+        """Raw queries of the shared instruction's tokens at one layer: [shared_len, Hq, D]."""
+        g = self.geom
+        return self._gen(Q_SHR, 0, (self.shared_len, g.n_q_heads, g.head_dim), layer * self.shared_len, device)
+
+    def ctx_q(self, b: int, layer: int, device="cpu") -> torch.Tensor:
+        """Raw queries of prompt b's context tokens at one layer: [L_b, Hq, D]."""
+        g = self.geom
+        L = int(self.ctx_len[b])
+        return self._gen(Q_CTX, b, (L, g.n_q_heads, g.head_dim), layer * L, device)
+
+    def question_q(self, k: int, layer: int, device="cpu") -> torch.Tensor:
+        """Raw queries of question k's own tokens at one layer: [n_k, Hq, D]."""
+        g = self.geom
+        n = int(self.q_len[k])
+        return self._gen(Q_QST, k, (n, g.n_q_heads, g.head_dim), layer * n, device)
 
     def _step_rows(self, kind: int, s: int, layer: int, qids, heads: int, device) -> torch.Tensor:
         g = self.geom

@@ -384,3 +384,65 @@ def test_layout_with_a_shared_instruction():
     assert lay["hdr_qtn_id"].tolist() == [0] * 5 + [0, 0, 0, 1, 1] + [0, 0, 2, 3, 3, 3]
     assert lay["hdr_begin"].tolist() == [5, 10, 16] and lay["ctx_tile_off"].tolist() == [1, 2, 3]
     assert orc.step_position(3, 2, 4, shared_len=5) == 14
+
+
+# ------------------------------------------------------------------ prefill of the stacked header
+def test_standalone_prefill_matches_library_causal_sdpa():
+    # library routine: torch SDPA with is_causal on an independently written complex-number RoPE
+    T, H, D, theta = 37, 3, 16, 1e4
+    r = np.random.default_rng(5)
+    k_raw, v_raw, q_raw = r.standard_normal((T, D)), r.standard_normal((T, D)), r.standard_normal((T, H, D))
+
+    def crope(x, pos):
+        z = x[..., : D // 2] + 1j * x[..., D // 2:]
+        w = np.exp(1j * pos * theta ** (-np.arange(D // 2) / (D / 2)))
+        zz = z * w
+        return np.concatenate([zz.real, zz.imag], axis=-1)
+
+    k = np.stack([crope(k_raw[i], i) for i in range(T)])
+    q = np.stack([crope(q_raw[i], i) for i in range(T)])  # [T, H, D]
+    want = torch.nn.functional.scaled_dot_product_attention(
+        torch.tensor(q).permute(1, 0, 2)[None], torch.tensor(k)[None, None].expand(1, H, T, D),
+        torch.tensor(v_raw)[None, None].expand(1, H, T, D), is_causal=True)[0].permute(1, 0, 2).numpy()
+    np.testing.assert_allclose(orc.standalone_prefill(k_raw, v_raw, q_raw, theta), want, atol=1e-12)
+    # its last row is the decode definition
+    np.testing.assert_allclose(orc.standalone_prefill(k_raw, v_raw, q_raw, theta)[-1],
+                               orc.standalone_attend(k_raw, v_raw, q_raw[-1], theta), atol=1e-12)
+
+
+@pytest.mark.parametrize("shared_len", [0, 4])
+def test_prefill_tuple_equals_header_rows_of_the_dense_formulation(shared_len):
+    # Sec. 4.1: under the dense mask a context token sees p and its own context causally, a question token sees p,
+    # its context and its own question prefix.  The header rows of dense_attend over the stacked sequence of the whole
+    # batch must equal the rows of the standalone prompts (p, c_b) and (p, c_b, x_k).
+    from paper_2609_05707_b200 import workloads as W
+    wl = W.custom_workload("pin4", W.Geometry(1, 4, 2, 16, 1e4), 79, [5, 3], [2, 1], [2, 3, 4], [1, 1, 1],
+                           shared_len=shared_len)
+    g, G, P = wl.geom, 2, wl.shared_len
+    q_lens = [[2, 3], [4]]
+    pos, ctx, qtn, tag = orc.stacked_sequence(P, [5, 3], q_lens, [[0, 0], [0]])
+    mask = orc.dense_mask(pos, ctx, qtn)
+    n = len(pos)
+    K, V, Q = np.zeros((n, 2, 16)), np.zeros((n, 2, 16)), np.zeros((n, 4, 16))
+    for i, (kind, j, kk, idx) in enumerate(tag):
+        k = int(wl.q_begin[j]) + kk
+        if kind == "p":
+            src = (wl.shared_kv(0), wl.shared_q(0))
+        elif kind == "c":
+            src = (wl.ctx_kv(j, 0), wl.ctx_q(j, 0))
+        else:
+            src = (wl.question_kv(k, 0), wl.question_q(k, 0))
+        K[i], V[i], Q[i] = src[0][0][idx].double().numpy(), src[0][1][idx].double().numpy(), src[1][idx].double().numpy()
+    dense = np.stack([orc.dense_attend(Q[:, h], np.repeat(K, G, axis=1)[:, h], np.repeat(V, G, axis=1)[:, h], pos, mask,
+                                       g.rope_theta) for h in range(4)], axis=1)  # [n, Hq, D]
+    for kv_head in range(2):
+        hs = slice(kv_head * G, (kv_head + 1) * G)
+        for b in range(2):
+            rows_c = [i for i, t in enumerate(tag) if t[0] == "c" and t[1] == b]
+            rows_p = [i for i, t in enumerate(tag) if t[0] == "p"]
+            got = orc.prefill_tuple(wl, b, None, 0, kv_head)
+            np.testing.assert_allclose(got, dense[rows_p + rows_c][:, hs], atol=1e-12, rtol=0)
+            for k in range(int(wl.q_begin[b]), int(wl.q_begin[b + 1])):
+                rows_x = [i for i, t in enumerate(tag) if t[0] == "x" and t[1] == b and t[2] == k - int(wl.q_begin[b])]
+                np.testing.assert_allclose(orc.prefill_tuple(wl, b, k, 0, kv_head), dense[rows_x][:, hs], atol=1e-12,
+                                           rtol=0)
