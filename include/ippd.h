@@ -54,6 +54,7 @@ extern "C" {
 #define IPPD_APPEND_QUESTION 1
 #define IPPD_APPEND_STEP 2
 #define IPPD_APPEND_SHARED 3
+#define IPPD_APPEND_HEADER 4
 
 /* keys of ippd_set_option */
 #define IPPD_OPT_KERNEL 1          /* 0 = auto, 1 = mma.sync path, 2 = tcgen05 path */
@@ -183,6 +184,9 @@ int ippd_step_descriptor_bytes(const ippd_layout_t* layout, const int32_t* activ
  * fp64-built table, result rounded to bf16) and store K and V into the cache
  * (paper Sec. 4.2, last paragraph: the token appended at each step carries its virtual position).
  *   kind SHARED  : ids ignored; tokens = the shared instruction's tokens (ippd_build_layout_shared), position i.
+ *   kind HEADER  : ids ignored; tokens = the whole stacked header in the order of the hdr_* tables (the shared
+ *                  instruction, then per prompt its context tokens and its questions' tokens), each at its
+ *                  virtual position: the whole prefill stand-in in one call.
  *   kind CONTEXT : ids[n_ids] = prompt ids (host); tokens = all context tokens of those
  *                  prompts, in id order; token i of prompt b gets position shared_len + i.
  *   kind QUESTION: ids[n_ids] = global question ids (host); tokens = their question
@@ -237,6 +241,28 @@ int ippd_decode_attention(ippd_layout_t* layout, int32_t layer_begin, int32_t la
 int ippd_decode_step(ippd_layout_t* layout, int32_t layer_begin, int32_t layer_count, const void* q_raw,
                      const void* k_raw, const void* v_raw, void* out, void* workspace,
                      size_t workspace_bytes, void* stream);
+
+/*
+ * ippd_prefill_attention -- the prefill of the stacked header under the IPPD mask (paper Sec. 4: the
+ * stacked prompt is prefilled once; Sec. 4.1: header rows of the mask; App. A.2: dim(q) of the prefill
+ * is the whole header).  Appends the header's K/V (as ippd_append_kv(HEADER)) and returns the
+ * attention output of EVERY header token:
+ *   instruction token i   sees instruction tokens 0..i;
+ *   context token i of b  sees the instruction and context tokens 0..i of its own prompt;
+ *   token j of question k sees the instruction, the context of its prompt and tokens 0..j of its question
+ * -- each row is the row of its own standalone causal prompt (Sec. 4.2).  q_raw: device bf16
+ * [layer_count, n_header_tokens, Hq, D]; k_raw, v_raw: [layer_count, n_header_tokens, Hkv, D] (pre-RoPE, header
+ * order of the hdr_* tables); out: [layer_count, n_header_tokens, Hq, D] in geom.out_dtype.  The same
+ * tensor-core kernel as the decode step runs it: 128-row blocks of consecutive header tokens stream
+ * the key tiles up to their own position, the diagonal tiles under per-row windows; question tokens
+ * see their question's prefix through packed branch pieces.  workspace as for ippd_decode_attention with
+ * layer_count layers.  Invalidates the step declared by ippd_begin_step.  Tensor-core path only.  The
+ * call allocates a device buffer for its work list (kept by the layout, reused by later calls).
+ * Errors: IPPD_ERR_INVALID_ARG, IPPD_ERR_NOT_BOUND, IPPD_ERR_OOM, IPPD_ERR_CUDA.
+ */
+int ippd_prefill_attention(ippd_layout_t* layout, int32_t layer_begin, int32_t layer_count, const void* q_raw,
+                           const void* k_raw, const void* v_raw, void* out, void* workspace,
+                           size_t workspace_bytes, void* stream);
 
 /*
  * ippd_decode_step_grouped -- ippd_decode_step for ALL layers of the step, `layers_per_call` layers per

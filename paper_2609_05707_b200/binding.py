@@ -21,11 +21,11 @@ OK, ERR_INVALID_ARG, ERR_OOM, ERR_CAPACITY, ERR_NOT_BOUND, ERR_CUDA, ERR_TIMEOUT
 BF16, F32 = 0, 1
 TILE_TOKENS = 128
 STATIC_SCRATCH_BYTES = 64 << 20
-APPEND_CONTEXT, APPEND_QUESTION, APPEND_STEP, APPEND_SHARED = 0, 1, 2, 3
+APPEND_CONTEXT, APPEND_QUESTION, APPEND_STEP, APPEND_SHARED, APPEND_HEADER = 0, 1, 2, 3, 4
 OPT_KERNEL, OPT_LAYERS_PER_CALL, OPT_TILES_PER_SPLIT, OPT_WAIT_LIMIT_US, OPT_PROFILE = 1, 2, 3, 4, 5
 
 EXPORTS = ["ippd_build_layout", "ippd_build_layout_shared", "ippd_layout_tables", "ippd_cache_bytes", "ippd_bind_cache", "ippd_set_option",
-           "ippd_begin_step", "ippd_step_descriptor_bytes", "ippd_append_kv", "ippd_workspace_bytes", "ippd_decode_attention", "ippd_decode_step", "ippd_decode_step_grouped", "ippd_decode_attention_static",
+           "ippd_begin_step", "ippd_step_descriptor_bytes", "ippd_append_kv", "ippd_workspace_bytes", "ippd_decode_attention", "ippd_decode_step", "ippd_decode_step_grouped", "ippd_prefill_attention", "ippd_decode_attention_static",
            "ippd_decode_step_host", "ippd_decode_step_host_async", "ippd_host_steps_wait", "ippd_step_stage_bytes", "ippd_export_mask", "ippd_poll_status", "ippd_profile_read", "ippd_read_probe", "ippd_host_time_read",
            "ippd_launch_count", "ippd_last_error", "ippd_destroy_layout"]
 
@@ -60,6 +60,7 @@ lib.ippd_append_kv.argtypes = [_vp, _i32, _i32, _i32, _pi32, _i32, _vp, _vp, _vp
 lib.ippd_workspace_bytes.argtypes = [_vp, _i32, C.POINTER(_sz)]
 lib.ippd_decode_attention.argtypes = [_vp, _i32, _i32, _vp, _vp, _vp, _sz, _vp]
 lib.ippd_decode_step.argtypes = [_vp, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
+lib.ippd_prefill_attention.argtypes = [_vp, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
 lib.ippd_decode_step_grouped.argtypes = [_vp, _i32, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
 lib.ippd_decode_attention_static.argtypes = [_vp, _i32, _i32, _vp, _vp, _vp]
 lib.ippd_decode_step_host.argtypes = [_vp, _pi32, _pi32, _i32, _vp, _vp, _vp, _vp, _vp, _sz, _vp, _sz, _vp]
@@ -194,6 +195,13 @@ class Layout:
         ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
         _check(lib.ippd_decode_step(self._h, layer_begin, layer_count, _dev(q_raw), _dev(k_raw), _dev(v_raw), _dev(out),
                                     _dev(workspace), ws_bytes, stream), "ippd_decode_step")
+
+    def prefill_attention(self, layer_begin: int, layer_count: int, q_raw, k_raw, v_raw, out, workspace,
+                          stream: int = 0):
+        """Prefill of the stacked header: appends its K/V and returns the attention output of every header token."""
+        ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+        _check(lib.ippd_prefill_attention(self._h, layer_begin, layer_count, _dev(q_raw), _dev(k_raw), _dev(v_raw),
+                                          _dev(out), _dev(workspace), ws_bytes, stream), "ippd_prefill_attention")
 
     def decode_step_grouped(self, layers_per_call: int, q_raw, k_raw, v_raw, out, workspace, stream: int = 0):
         """decode_step for all layers of the step, `layers_per_call` layers per launch."""

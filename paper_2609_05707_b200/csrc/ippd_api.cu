@@ -33,7 +33,10 @@ struct ippd_layout {
   int device = -1;
   // device mirrors
   int32_t *d_ctx_len = nullptr, *d_ctx_tile_off = nullptr, *d_q_len = nullptr, *d_prompt_of = nullptr,
-          *d_branch_tile_off = nullptr, *d_error = nullptr;
+          *d_branch_tile_off = nullptr, *d_error = nullptr, *d_hdr_begin = nullptr, *d_q_hdr_begin = nullptr,
+          *d_q_first = nullptr;
+  char* prefill_dev = nullptr;  // device copy of the prefill's work list
+  size_t prefill_cap = 0;
   float2* d_rope = nullptr;
   char* cache = nullptr;
   // ring of pinned host / device slots for the small per-call descriptors
@@ -158,6 +161,8 @@ static IppdDev make_dev(const ippd_layout* L) {
   d.q_len = L->d_q_len;
   d.prompt_of = L->d_prompt_of;
   d.branch_tile_off = L->d_branch_tile_off;
+  d.hdr_begin = L->d_hdr_begin;
+  d.q_hdr_begin = L->d_q_hdr_begin;
   d.rope = L->d_rope;
   d.cache = L->cache;
   d.error_word = L->d_error;
@@ -268,6 +273,10 @@ static int upload_vec(T** dst, const std::vector<T>& v) {
 static void free_device(ippd_layout* L) {
   cudaFree(L->d_ctx_len); cudaFree(L->d_ctx_tile_off); cudaFree(L->d_q_len); cudaFree(L->d_prompt_of);
   cudaFree(L->d_branch_tile_off); cudaFree(L->d_error); cudaFree(L->d_rope);
+  cudaFree(L->d_hdr_begin); cudaFree(L->d_q_hdr_begin); cudaFree(L->d_q_first); cudaFree(L->prefill_dev);
+  L->d_hdr_begin = L->d_q_hdr_begin = L->d_q_first = nullptr;
+  L->prefill_dev = nullptr;
+  L->prefill_cap = 0;
   L->d_ctx_len = L->d_ctx_tile_off = L->d_q_len = L->d_prompt_of = L->d_branch_tile_off = L->d_error = nullptr;
   L->d_rope = nullptr;
   for (int i = 0; i < kRingSlots; ++i) {
@@ -296,6 +305,18 @@ extern "C" int ippd_bind_cache(ippd_layout_t* L, void* dev_cache, size_t bytes, 
   if ((rc = upload_vec(&L->d_q_len, h.q_len)) != IPPD_OK) return rc;
   if ((rc = upload_vec(&L->d_prompt_of, h.prompt_of)) != IPPD_OK) return rc;
   if ((rc = upload_vec(&L->d_branch_tile_off, h.branch_tile_off)) != IPPD_OK) return rc;
+  {
+    // header offsets: first header token of each prompt and of each question (the hdr_* order)
+    std::vector<int32_t> hb(h.hdr_begin.begin(), h.hdr_begin.end()), qb((size_t)h.NQ + 1, 0);
+    for (int b = 0; b < h.B; ++b) {
+      int64_t t = h.hdr_begin[b] + h.ctx_len[b];
+      for (int k = h.q_begin[b]; k < h.q_begin[b + 1]; ++k) { qb[k] = (int32_t)t; t += h.q_len[k]; }
+    }
+    qb[h.NQ] = (int32_t)h.hdr_begin[h.B];
+    if ((rc = upload_vec(&L->d_hdr_begin, hb)) != IPPD_OK) return rc;
+    if ((rc = upload_vec(&L->d_q_hdr_begin, qb)) != IPPD_OK) return rc;
+    if ((rc = upload_vec(&L->d_q_first, h.q_begin)) != IPPD_OK) return rc;
+  }
   CUDA_TRY(cudaMalloc((void**)&L->d_error, sizeof(int32_t)));
   CUDA_TRY(cudaMemset(L->d_error, 0, sizeof(int32_t)));
   size_t n_rope = (size_t)(h.max_pos + 1) * (h.geom.head_dim / 2);
@@ -400,13 +421,9 @@ extern "C" int ippd_begin_step(ippd_layout_t* L, const int32_t* active_q, const 
     memcpy(blob.data() + off_tb, P.rb_tile_begin.data(), P.rb_tile_begin.size() * 4);
     if (!P.tc_tiles.empty()) memcpy(blob.data() + off_tt, P.tc_tiles.data(), P.tc_tiles.size() * sizeof(IppdTcTile));
     if (!P.tc_pieces.empty()) memcpy(blob.data() + off_tp, P.tc_pieces.data(), P.tc_pieces.size() * sizeof(IppdTcPiece));
-    // virtual position of every active question's query (Sec. 4.1): context length + question length + answer index;
-    // kept in the descriptor so that the kernels' Q~ staging does not chase it through three tables
-    int32_t* pos = reinterpret_cast<int32_t*>(blob.data() + off_pos);
-    for (int a = 0; a < A; ++a) {
-      const int k = P.act_q[a];
-      pos[a] = L->h.shared_len + L->h.ctx_len[L->h.prompt_of[k]] + L->h.q_len[k] + P.act_s[a];
-    }
+    // virtual position of every query (Sec. 4.1), kept in the descriptor so that the kernels' Q~ staging does not
+    // chase it through three tables
+    memcpy(blob.data() + off_pos, P.act_pos.data(), (size_t)A * 4);
   }
   char* dev = nullptr;
   L->pending_slot = -1;  // a step that was declared but never used is dropped
@@ -482,8 +499,10 @@ extern "C" int ippd_append_kv(ippd_layout_t* L, int32_t layer_begin, int32_t lay
       int rc = ring_flush(L, stream);
       if (rc != IPPD_OK) return rc;
     }
-  } else if (kind == IPPD_APPEND_SHARED) {
-    a.n_tokens = h.shared_len;
+  } else if (kind == IPPD_APPEND_SHARED || kind == IPPD_APPEND_HEADER) {
+    a.n_tokens = kind == IPPD_APPEND_SHARED ? h.shared_len : (int)h.hdr_pos.size();
+    a.n_ids = h.B;
+    a.q_first = L->d_q_first;
     int rc = ring_flush(L, stream);  // keeps the descriptor ring in stream order
     if (rc != IPPD_OK) return rc;
   } else if (kind == IPPD_APPEND_CONTEXT || kind == IPPD_APPEND_QUESTION) {
@@ -817,6 +836,94 @@ extern "C" int ippd_decode_attention_static(ippd_layout_t* L, int32_t layer_begi
   if (h.geom.head_dim == 128)
     return launch_attention<128>(L, d, layer_begin, layer_count, q_raw, out, part_o, part_ml, stream, false);
   return launch_attention<64>(L, d, layer_begin, layer_count, q_raw, out, part_o, part_ml, stream, false);
+}
+
+extern "C" int ippd_prefill_attention(ippd_layout_t* L, int32_t layer_begin, int32_t layer_count, const void* q_raw,
+                                      const void* k_raw, const void* v_raw, void* out, void* workspace,
+                                      size_t workspace_bytes, void* stream_) {
+  if (!L) { ippd_set_error("ippd_prefill_attention: NULL layout"); return IPPD_ERR_INVALID_ARG; }
+  if (!L->bound) { ippd_set_error("ippd_prefill_attention: no cache bound"); return IPPD_ERR_NOT_BOUND; }
+  const IppdHostLayout& h = L->h;
+  if (h.kernel_path() != 2) { ippd_set_error("ippd_prefill_attention: tensor-core path only"); return IPPD_ERR_INVALID_ARG; }
+  if (layer_begin < 0 || layer_count < 1 || layer_begin + layer_count > h.geom.n_layers) {
+    ippd_set_error("ippd_prefill_attention: layer range out of bounds");
+    return IPPD_ERR_INVALID_ARG;
+  }
+  if (!q_raw || !k_raw || !v_raw || !out) { ippd_set_error("ippd_prefill_attention: NULL tensor"); return IPPD_ERR_INVALID_ARG; }
+  cudaStream_t stream = (cudaStream_t)stream_;
+  const int n_hdr = (int)h.hdr_pos.size();
+  if (n_hdr == 0) return IPPD_OK;
+  // 1. the header's K/V into the cache
+  int rc = ippd_append_kv(L, layer_begin, layer_count, IPPD_APPEND_HEADER, nullptr, 0, k_raw, v_raw, stream_);
+  if (rc != IPPD_OK) return rc;
+  // 2. one query per header token, in header order
+  std::vector<IppdPlanEntry> ent((size_t)n_hdr);
+  int t = 0;
+  for (; t < h.shared_len; ++t) ent[t] = {-1, -1, 0, 1};
+  for (int b = 0; b < h.B; ++b) {
+    for (int i = 0; i < h.ctx_len[b]; ++i, ++t) ent[t] = {b, -1, 0, 1};
+    for (int k = h.q_begin[b]; k < h.q_begin[b + 1]; ++k)
+      for (int j = 0; j < h.q_len[k]; ++j, ++t) ent[t] = {b, k, j + 1, 0};
+  }
+  L->have_step = false;
+  L->pending_slot = -1;
+  L->profile = L->profile_stride > 0;
+  rc = ippd_host_plan_entries(h, ent.data(), h.hdr_pos.data(), n_hdr, layer_count, false, &L->plan);
+  if (rc != IPPD_OK) return rc;
+  const IppdStepPlan& P = L->plan;
+  const StepBlobLayout bl = step_blob_layout((size_t)n_hdr, P.rbs.size(), P.units.size(), P.tc_tiles.size(), P.tc_pieces.size());
+  std::vector<char> blob(bl.total, 0);
+  memcpy(blob.data() + bl.off_rb, P.rbs.data(), P.rbs.size() * sizeof(IppdRowBlock));
+  memcpy(blob.data() + bl.off_tb, P.rb_tile_begin.data(), P.rb_tile_begin.size() * 4);
+  memcpy(blob.data() + bl.off_tt, P.tc_tiles.data(), P.tc_tiles.size() * sizeof(IppdTcTile));
+  if (!P.tc_pieces.empty()) memcpy(blob.data() + bl.off_tp, P.tc_pieces.data(), P.tc_pieces.size() * sizeof(IppdTcPiece));
+  memcpy(blob.data() + bl.off_pos, P.act_pos.data(), (size_t)n_hdr * 4);
+  if (bl.total > L->prefill_cap) {
+    CUDA_TRY(cudaStreamSynchronize(stream));  // an earlier prefill may still read the old buffer
+    cudaFree(L->prefill_dev);
+    L->prefill_dev = nullptr;
+    L->prefill_cap = 0;
+    if (cudaMalloc((void**)&L->prefill_dev, bl.total) != cudaSuccess) { ippd_set_error("ippd_prefill_attention: out of device memory"); return IPPD_ERR_OOM; }
+    L->prefill_cap = bl.total;
+  }
+  CUDA_TRY(cudaMemcpyAsync(L->prefill_dev, blob.data(), bl.total, cudaMemcpyHostToDevice, stream));
+  CUDA_TRY(cudaStreamSynchronize(stream));  // `blob` is pageable host memory of this call
+  char* dev = L->prefill_dev;
+  L->step_dev.act_q = (const int32_t*)(dev + bl.off_q);
+  L->step_dev.act_s = (const int32_t*)(dev + bl.off_s);
+  L->step_dev.rbs = (const IppdRowBlock*)(dev + bl.off_rb);
+  L->step_dev.act_pos = (const int32_t*)(dev + bl.off_pos);
+  L->step_dev.units = (const IppdUnit*)(dev + bl.off_u);
+  L->d_rb_tile_begin = (const int32_t*)(dev + bl.off_tb);
+  L->d_tc_tiles = (const IppdTcTile*)(dev + bl.off_tt);
+  L->d_tc_pieces = (const IppdTcPiece*)(dev + bl.off_tp);
+  L->step_dev.A = n_hdr;
+  L->step_dev.n_rb = P.hdr.n_rowblocks;
+  L->step_dev.n_units = 0;
+  L->step_dev.RB = P.hdr.rows_per_block;
+  L->last_stream = stream;
+  // 3. the attention pass
+  L->have_step = true;
+  size_t o_bytes = 0;
+  bool needed = false;
+  const size_t need = scratch_need(L, layer_count, &o_bytes, &needed);
+  float *part_o = nullptr, *part_ml = nullptr;
+  if (needed) {
+    if (!workspace || workspace_bytes < need || (uintptr_t)workspace % 256 != 0) {
+      L->have_step = false;
+      ippd_set_error("ippd_prefill_attention: workspace missing, misaligned or too small");
+      return IPPD_ERR_INVALID_ARG;
+    }
+    part_o = (float*)workspace;
+    part_ml = (float*)((char*)workspace + o_bytes);
+  }
+  IppdDev d = make_dev(L);
+  rc = h.geom.head_dim == 128
+           ? launch_attention<128>(L, d, layer_begin, layer_count, q_raw, out, part_o, part_ml, stream, true)
+           : launch_attention<64>(L, d, layer_begin, layer_count, q_raw, out, part_o, part_ml, stream, true);
+  L->have_step = false;  // the work list in force is the prefill's: a decode step must be declared anew
+  L->profile = false;
+  return rc;
 }
 
 extern "C" int ippd_decode_step_grouped(ippd_layout_t* L, int32_t layers_per_call, const void* q_raw, const void* k_raw,

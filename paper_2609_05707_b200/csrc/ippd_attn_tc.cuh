@@ -307,6 +307,7 @@ ippd_attn_tc_kernel(IppdDev L, IppdStepDev S, IppdTcArgs A, const __nv_bfloat16*
     bool ok = true;
     while (ok && tc_next_segment(A, S, Hkv, g0, g1, g, sg)) {
       const int layer = A.layer_begin + sg.ll;
+      const int seg_act_begin = S.rbs[sg.rb].act_begin, seg_n_act = S.rbs[sg.rb].n_act;
       for (int t = sg.t_begin; t < sg.t_end && ok; ++t, ++tc) {
         const IppdTcTile ti = A.tiles[t];
         IppdTcPiece pc;
@@ -325,6 +326,15 @@ ippd_attn_tc_kernel(IppdDev L, IppdStepDev S, IppdTcArgs A, const __nv_bfloat16*
           if (lane < ti.n_pieces) {
             if (lane == 0 || a_prev != a_me) mt.c0[a_me] = (uint8_t)pc.row0;
             if (lane == ti.n_pieces - 1 || a_next != a_me) mt.c1[a_me] = (uint8_t)(pc.row0 + pc.valid);
+          }
+        } else if (ti.n_pieces < 0) {
+          // causal context tile (prefill): query a of the row block sits at virtual position pos_a and sees the
+          // tile's tokens up to itself, columns [0, pos_a + 1 - first position of the tile)
+          for (int a = lane; a < 64; a += 32) {
+            int c1 = 0;
+            if (a < seg_n_act) c1 = max(0, min(ti.rows, S.act_pos[seg_act_begin + a] + 1 - ti.piece_begin));
+            mt.c0[a] = 0;
+            mt.c1[a] = (uint8_t)c1;
           }
         }
         __syncwarp();
@@ -351,7 +361,7 @@ ippd_attn_tc_kernel(IppdDev L, IppdStepDev S, IppdTcArgs A, const __nv_bfloat16*
           }
           if (lane == 0) mbar_arrive_expect_tx(&sh->kv_full[buf], (uint32_t)groups * GB);
           __syncwarp();
-          if (ti.n_pieces == 0) {
+          if (ti.n_pieces <= 0) {
             if (lane == 0)
               bulk_g2s(dst, L.cache + ippd_tile_addr(L, layer, sg.head, ti.pool_tile, kv), (uint32_t)groups * GB,
                        &sh->kv_full[buf]);

@@ -72,6 +72,7 @@ struct IppdAppendArgs {
   int n_ids;
   const int32_t* ids;        // device: prompt or question ids (CONTEXT / QUESTION)
   const int32_t* tok_begin;  // device: [n_ids+1] first token of each id
+  const int32_t* q_first;    // device: [B+1] first question of each prompt (HEADER)
   // STEP appends of at most IPPD_APPEND_INLINE tokens carry the step's active list in the kernel parameters and also
   // move the step's descriptor from its pinned slot to the device (blocks past the first n_append_blocks of row 0):
   // the append does not have to wait for a separate upload kernel, and the upload's PCIe latency hides behind it.
@@ -115,10 +116,33 @@ ippd_append_kernel(IppdDev L, IppdStepDev S, IppdAppendArgs a, int layer_begin,
     pos = L.shared_len + L.ctx_len[L.prompt_of[qid]] + slot;
     tile = L.branch_tile_off[qid] + slot / IPPD_TILE_TOKENS;
     u = slot % IPPD_TILE_TOKENS;
-  } else if (a.kind == IPPD_APPEND_SHARED) {
+  } else if (a.kind == IPPD_APPEND_SHARED || (a.kind == IPPD_APPEND_HEADER && tok < L.shared_len)) {
     pos = tok;
     tile = tok / IPPD_TILE_TOKENS;
     u = tok % IPPD_TILE_TOKENS;
+  } else if (a.kind == IPPD_APPEND_HEADER) {
+    // token `tok` of the stacked header: find its prompt, then whether it is a context or a question token
+    int lo = 0, hi = a.n_ids - 1;  // n_ids = number of prompts
+    while (lo < hi) {
+      int mid = (lo + hi + 1) >> 1;
+      if (L.hdr_begin[mid] <= tok) lo = mid; else hi = mid - 1;
+    }
+    const int b = lo, i = tok - L.hdr_begin[b];
+    if (i < L.ctx_len[b]) {
+      pos = L.shared_len + i;
+      tile = L.ctx_tile_off[b] + i / IPPD_TILE_TOKENS;
+      u = i % IPPD_TILE_TOKENS;
+    } else {
+      int qlo = a.q_first[b], qhi = a.q_first[b + 1] - 1;  // questions of prompt b
+      while (qlo < qhi) {
+        int mid = (qlo + qhi + 1) >> 1;
+        if (L.q_hdr_begin[mid] <= tok) qlo = mid; else qhi = mid - 1;
+      }
+      const int j = tok - L.q_hdr_begin[qlo];
+      pos = L.shared_len + L.ctx_len[b] + j;
+      tile = L.branch_tile_off[qlo] + j / IPPD_TILE_TOKENS;
+      u = j % IPPD_TILE_TOKENS;
+    }
   } else {
     int lo = 0, hi = a.n_ids - 1;  // last id whose first token is <= tok
     while (lo < hi) {

@@ -17,6 +17,8 @@ struct IppdDev {
   const int32_t* q_len;            // [NQ]
   const int32_t* prompt_of;        // [NQ]
   const int32_t* branch_tile_off;  // [NQ+1]
+  const int32_t* hdr_begin;        // [B+1] first header token of each prompt (the shared instruction comes first)
+  const int32_t* q_hdr_begin;      // [NQ+1] first header token of each question
   const float2* rope;              // [max_pos+1][D/2] (cos, sin)
   char* cache;                     // [layer][kv head][tile][K|V][tile bytes]
   int32_t* error_word;

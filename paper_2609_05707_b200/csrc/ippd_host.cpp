@@ -153,10 +153,37 @@ int ippd_host_plan_step(const IppdHostLayout& L, const int32_t* active_q, const 
     ippd_set_error("ippd_begin_step: bad active list");
     return IPPD_ERR_INVALID_ARG;
   }
-  const int RB = L.rows_per_block();
-  const int qpr = questions_per_block(L);
+  static thread_local std::vector<IppdPlanEntry> ent;
+  static thread_local std::vector<int32_t> pos;
+  ent.resize(A);
+  pos.resize(A);
+  int32_t prev = -1;
+  for (int a = 0; a < A; ++a) {
+    const int32_t k = active_q[a];
+    if (k < 0 || k >= L.NQ) { ippd_set_error("ippd_begin_step: question id out of range"); return IPPD_ERR_INVALID_ARG; }
+    if (k <= prev) { ippd_set_error("ippd_begin_step: active_q must be strictly increasing"); return IPPD_ERR_INVALID_ARG; }
+    if (answer_idx[a] < 0) { ippd_set_error("ippd_begin_step: answer_idx < 0"); return IPPD_ERR_INVALID_ARG; }
+    if (answer_idx[a] >= L.max_new[k]) { ippd_set_error("ippd_begin_step: answer_idx >= max_new (branch capacity)"); return IPPD_ERR_CAPACITY; }
+    prev = k;
+    const int b = L.prompt_of[k];
+    ent[a] = {b, k, L.q_len[k] + answer_idx[a] + 1, 0};
+    // virtual position of the query (Sec. 4.1): instruction + context + question length + answer index
+    pos[a] = L.shared_len + L.ctx_len[b] + L.q_len[k] + answer_idx[a];
+  }
+  int rc = ippd_host_plan_entries(L, ent.data(), pos.data(), A, layer_count, true, plan);
+  if (rc != IPPD_OK) return rc;
   plan->act_q.assign(active_q, active_q + A);
   plan->act_s.assign(answer_idx, answer_idx + A);
+  return IPPD_OK;
+}
+
+int ippd_host_plan_entries(const IppdHostLayout& L, const IppdPlanEntry* ent, const int32_t* pos, int32_t A,
+                           int32_t layer_count, bool mark_new, IppdStepPlan* plan) {
+  const int RB = L.rows_per_block();
+  const int qpr = questions_per_block(L);
+  plan->act_q.assign(A, 0);
+  plan->act_s.assign(A, 0);
+  plan->act_pos.assign(pos, pos + A);
   plan->rbs.clear();
   plan->units.clear();
   plan->tc_tiles.clear();
@@ -168,37 +195,49 @@ int ippd_host_plan_step(const IppdHostLayout& L, const int32_t* active_q, const 
   }
   int64_t total = 0;
   int i = 0;
-  int32_t prev = -1;
   while (i < A) {
-    int32_t k0 = active_q[i];
-    if (k0 < 0 || k0 >= L.NQ) { ippd_set_error("ippd_begin_step: question id out of range"); return IPPD_ERR_INVALID_ARG; }
-    int b = L.prompt_of[k0];
+    const int b = ent[i].prompt;
+    const int causal = ent[i].causal;
     int j = i;
-    while (j < A && active_q[j] < L.q_begin[b + 1]) {
-      int32_t k = active_q[j];
-      if (k <= prev) { ippd_set_error("ippd_begin_step: active_q must be strictly increasing"); return IPPD_ERR_INVALID_ARG; }
-      if (answer_idx[j] < 0) { ippd_set_error("ippd_begin_step: answer_idx < 0"); return IPPD_ERR_INVALID_ARG; }
-      if (answer_idx[j] >= L.max_new[k]) { ippd_set_error("ippd_begin_step: answer_idx >= max_new (branch capacity)"); return IPPD_ERR_CAPACITY; }
-      prev = k;
-      ++j;
+    while (j < A && ent[j].prompt == b && ent[j].causal == causal) ++j;
+    if (!tc_path && (causal || b < 0)) {
+      ippd_set_error("prefill needs the tensor-core path (IPPD_OPT_KERNEL 0 or 2)");
+      return IPPD_ERR_INVALID_ARG;
     }
-    const int nct_own = L.ctx_tile_off[b + 1] - L.ctx_tile_off[b];
-    const int nct = L.n_shared_tiles + nct_own;  // every query row sees the shared instruction, then its own context
+    const int nct_own = b >= 0 ? L.ctx_tile_off[b + 1] - L.ctx_tile_off[b] : 0;
     for (int a0 = i; a0 < j; a0 += qpr) {
       IppdRowBlock rb;
       memset(&rb, 0, sizeof(rb));
       rb.prompt = b;
       rb.act_begin = a0;
       rb.n_act = std::min(qpr, j - a0);
+      // every query row sees the shared instruction, then its own context; a causal row only up to its own position
+      int n_sh = L.n_shared_tiles, n_own = nct_own;
+      int pos_min = 0;
+      if (causal) {
+        int pos_max = 0;
+        pos_min = INT_MAX;
+        for (int a = a0; a < a0 + rb.n_act; ++a) { pos_max = std::max(pos_max, pos[a]); pos_min = std::min(pos_min, pos[a]); }
+        if (pos_max < L.shared_len) {
+          n_sh = pos_max / IPPD_TILE_TOKENS + 1;
+          n_own = 0;
+        } else {
+          n_own = std::min(nct_own, (pos_max - L.shared_len) / IPPD_TILE_TOKENS + 1);
+        }
+      }
+      const int nct = n_sh + n_own;
       rb.n_ctx_tiles = nct;
       int64_t tiles = nct;
       if (tc_path) {
-        for (int t = 0; t < L.n_shared_tiles; ++t) {
+        for (int t = 0; t < n_sh; ++t) {
           IppdTcTile ti = {t, std::min(IPPD_TILE_TOKENS, L.shared_len - t * IPPD_TILE_TOKENS), 0, 0};
+          if (causal && t * IPPD_TILE_TOKENS + ti.rows - 1 >= pos_min) { ti.n_pieces = -1; ti.piece_begin = t * IPPD_TILE_TOKENS; }
           plan->tc_tiles.push_back(ti);
         }
-        for (int t = 0; t < nct_own; ++t) {
+        for (int t = 0; t < n_own; ++t) {
           IppdTcTile ti = {L.ctx_tile_off[b] + t, std::min(IPPD_TILE_TOKENS, L.ctx_len[b] - t * IPPD_TILE_TOKENS), 0, 0};
+          const int tok0 = L.shared_len + t * IPPD_TILE_TOKENS;  // virtual position of the tile's first token
+          if (causal && tok0 + ti.rows - 1 >= pos_min) { ti.n_pieces = -1; ti.piece_begin = tok0; }
           plan->tc_tiles.push_back(ti);
         }
         // Pack the branches of the block's questions, 8-token group by group, into 128-row tiles.  Every tile takes
@@ -218,12 +257,12 @@ int ippd_host_plan_step(const IppdHostLayout& L, const int32_t* active_q, const 
           runs[qu].clear();
           const int a_end = std::min(a0 + rb.n_act, a0 + (qu + 1) * q_per_quarter);
           for (int a = a0 + qu * q_per_quarter; a < a_end; ++a) {
-            const int k = active_q[a];
-            const int len = L.q_len[k] + answer_idx[a] + 1;
+            const int k = ent[a].branch;
+            const int len = k >= 0 ? ent[a].branch_len : 0;
             for (int jt = 0; jt * IPPD_TILE_TOKENS < len; ++jt) {
               const int valid_j = std::min(IPPD_TILE_TOKENS, len - jt * IPPD_TILE_TOKENS);
               runs[qu].push_back({a - a0, L.branch_tile_off[k] + jt, 0, (valid_j + 7) / 8, valid_j,
-                                  (jt + 1) * IPPD_TILE_TOKENS >= len});
+                                  mark_new && (jt + 1) * IPPD_TILE_TOKENS >= len});
               rem[qu] += (valid_j + 7) / 8;
             }
           }
@@ -273,7 +312,7 @@ int ippd_host_plan_step(const IppdHostLayout& L, const int32_t* active_q, const 
         }
       } else {
         for (int a = a0; a < a0 + rb.n_act; ++a)
-          tiles += ceil_div((int64_t)L.q_len[active_q[a]] + answer_idx[a] + 1, IPPD_TILE_TOKENS);
+          tiles += ceil_div((int64_t)ent[a].branch_len, IPPD_TILE_TOKENS);
       }
       rb.n_tiles = (int32_t)tiles;
       rb.tile_begin = (int32_t)total;
@@ -315,10 +354,6 @@ int ippd_host_plan_step(const IppdHostLayout& L, const int32_t* active_q, const 
       plan->units.push_back(u);
     }
   }
-  plan->total_tiles = total;
-  plan->hdr.n_active = A;
-  plan->hdr.n_rowblocks = (int32_t)plan->rbs.size();
   plan->hdr.n_units = (int32_t)plan->units.size();
-  plan->hdr.rows_per_block = RB;
   return IPPD_OK;
 }

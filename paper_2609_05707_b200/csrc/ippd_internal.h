@@ -39,6 +39,8 @@ struct IppdUnit {
 
 // Key tile of the tensor-core path.  A context tile (n_pieces == 0) is pool tile `pool_tile` with `rows` valid tokens.
 // A packed branch tile (n_pieces > 0) is the concatenation of pieces; `rows` = 8 x the groups it holds.
+// A causal context tile (n_pieces == -1, prefill only) is a context tile of which a query row sees only the tokens up
+// to its own position; piece_begin then holds the virtual position of the tile's first token.
 struct IppdTcTile {
   int32_t pool_tile;
   int32_t rows;
@@ -57,9 +59,17 @@ struct IppdTcPiece {
   int32_t pad1;
 };
 
+// One query of a planned pass: a decode step's token, or a header token of the prefill.
+struct IppdPlanEntry {
+  int32_t prompt;      // -1: a token of the shared instruction
+  int32_t branch;      // question whose branch the query sees, -1: none
+  int32_t branch_len;  // how many of the branch's tokens it sees (from slot 0)
+  int32_t causal;      // 1: of the (instruction, context) key stream it sees only the tokens up to its own position
+};
+
 struct IppdStepPlan {
   IppdStepHeader hdr;
-  std::vector<int32_t> act_q, act_s;
+  std::vector<int32_t> act_q, act_s, act_pos;
   std::vector<IppdRowBlock> rbs;
   std::vector<IppdUnit> units;
   std::vector<int32_t> rb_tile_begin;  // [n_rb+1] prefix sums of n_tiles
@@ -98,6 +108,10 @@ int ippd_host_build(const ippd_geometry_t* geom, int32_t shared_len, int32_t n_p
 // Builds the work list of one step.  Returns IPPD_OK or an error code.
 int ippd_host_plan_step(const IppdHostLayout& L, const int32_t* active_q, const int32_t* answer_idx,
                         int32_t n_active, int32_t layer_count, IppdStepPlan* plan);
+// The same for an arbitrary list of queries (consecutive entries of one prompt and one kind form row blocks);
+// pos[i] = virtual position of entry i; mark_new: the last visible branch token of every entry is the step's new token.
+int ippd_host_plan_entries(const IppdHostLayout& L, const IppdPlanEntry* ent, const int32_t* pos, int32_t n,
+                           int32_t layer_count, bool mark_new, IppdStepPlan* plan);
 // Upper bound of plan.units.size() over all possible steps.
 int64_t ippd_host_max_units(const IppdHostLayout& L, int32_t layer_count);
 int64_t ippd_host_max_rowblocks(const IppdHostLayout& L);

@@ -45,7 +45,7 @@ ippd_read_probe_kernel(IppdDev L, IppdStepDev S, IppdTcArgs A) {
         uint8_t* dst = ring + buf * TILE_BYTES;
         if (lane == 0) mbar_arrive_expect_tx(&full[buf], (uint32_t)groups * GB);
         __syncwarp();
-        if (ti.n_pieces == 0) {
+        if (ti.n_pieces <= 0) {
           if (lane == 0)
             bulk_g2s(dst, L.cache + ippd_tile_addr(L, layer, sg.head, ti.pool_tile, kv), (uint32_t)groups * GB, &full[buf]);
         } else if (lane < ti.n_pieces) {

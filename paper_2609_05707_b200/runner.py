@@ -74,6 +74,47 @@ class Runner:
                                   torch.cat(vs).contiguous(), self.stream)
         torch.cuda.synchronize(self.device)
 
+    def header_inputs(self, layer: int):
+        """Raw q, k, v of every header token at one layer, in the order of the layout's hdr_* tables (the shared
+        instruction, then per prompt its context tokens and its questions' tokens): [n_hdr, H, D] each."""
+        wl, dev = self.wl, self.device
+        qs, ks, vs = [], [], []
+        if wl.shared_len > 0:
+            k, v = wl.shared_kv(layer, dev)
+            qs.append(wl.shared_q(layer, dev)); ks.append(k); vs.append(v)
+        for b in range(wl.n_prompts):
+            if wl.ctx_len[b] > 0:
+                k, v = wl.ctx_kv(b, layer, dev)
+                qs.append(wl.ctx_q(b, layer, dev)); ks.append(k); vs.append(v)
+            for qid in range(int(wl.q_begin[b]), int(wl.q_begin[b + 1])):
+                k, v = wl.question_kv(qid, layer, dev)
+                qs.append(wl.question_q(qid, layer, dev)); ks.append(k); vs.append(v)
+        return torch.cat(qs).contiguous(), torch.cat(ks).contiguous(), torch.cat(vs).contiguous()
+
+    def prefill(self, layers_per_call: int = 1, keep_out: bool = True):
+        """Prefill of the stacked header through ippd_prefill_attention, `layers_per_call` layers per call: fills the
+        cache with the header's K/V and returns the attention output of every header token,
+        [n_layers, n_hdr, Hq, D] (None when keep_out is False)."""
+        g = self.wl.geom
+        need = self.layout.workspace_bytes(layers_per_call)
+        if need > self.workspace.numel():
+            self.workspace = self.alloc_bytes(need, "workspace")
+        outs = []
+        for l0 in range(0, g.n_layers, layers_per_call):
+            n = min(layers_per_call, g.n_layers - l0)
+            qkv = [self.header_inputs(l) for l in range(l0, l0 + n)]
+            q = torch.stack([t[0] for t in qkv]).contiguous()
+            k = torch.stack([t[1] for t in qkv]).contiguous()
+            v = torch.stack([t[2] for t in qkv]).contiguous()
+            shape = (n, q.shape[1], g.n_q_heads, g.head_dim)
+            nbytes = int(np.prod(shape)) * (4 if self.out_torch_dtype == torch.float32 else 2)
+            out = self.alloc_bytes(nbytes, "out").view(self.out_torch_dtype).view(shape)
+            self.layout.prefill_attention(l0, n, q, k, v, out, self.workspace, self.stream)
+            torch.cuda.synchronize(self.device)
+            if keep_out:
+                outs.append(out)
+        return torch.cat(outs) if keep_out else None
+
     # ------------------------------------------------------------------ decode
     def step_inputs(self, s: int, act: np.ndarray):
         """Raw q, k, v of step s for the active questions, all layers: [layers, A, H, D] each."""

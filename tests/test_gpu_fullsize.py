@@ -43,12 +43,13 @@ def run_and_sample(name, check, per_prompt, kernel=0, full_layer_step=None):
     G = wl.geom.group
     run = PoisonedRunner(wl, kernel=kernel)
     run.load_header()
+    # the K/V of every step go into the cache first (a token's slot depends only on its question and step index, and a
+    # step reads no slot beyond its own), then only the sampled steps are run; each of them appends its own token again
+    run.append_all_steps()
     ctx_cache, step_cache = {}, {}
     n_tuples = 0
-    for s in range(max(check) + 1):
+    for s in sorted(check):
         act, out = run.run_step(s)
-        if s not in check:
-            continue
         run.check()
         rows = {int(k): i for i, k in enumerate(act)}
         for layer, head in check[s]:
