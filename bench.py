@@ -202,12 +202,12 @@ def spread_steps(n_steps: int, count: int):
 class ConfigBench:
     """One workload resident on the device, every step's K/V already in the cache."""
 
-    def __init__(self, name, dev, kernel, max_resident_bytes=24e9):
+    def __init__(self, name, dev, kernel, max_resident_bytes=24e9, n_layers=0):
         import torch
         from paper_2609_05707_b200 import workloads as W
         from paper_2609_05707_b200.runner import Runner
         self.torch = torch
-        self.wl = wl = W.make_workload(name)
+        self.wl = wl = W.make_workload(name, n_layers or None)
         self.g = g = wl.geom
         self.dev = dev
         self.run = Runner(wl, dev, kernel=kernel, layers_per_call=g.n_layers)
@@ -273,6 +273,57 @@ class ConfigBench:
         lay.set_option(B.OPT_PROFILE, 0)
         return prof
 
+    def prefill(self, peaks, layers=2, reps=2):
+        """ippd_prefill_attention over the first `layers` layers of the stacked header: device time per layer and the
+        fraction of the sustained bf16 tensor peak (the prefill is a dense contraction: every 128-row block of header
+        tokens streams all key tiles up to its own position)."""
+        from paper_2609_05707_b200 import binding as B
+        torch = self.torch
+        run, wl, g = self.run, self.wl, self.g
+        layers = min(layers, g.n_layers)
+        qkv = [run.header_inputs(l) for l in range(layers)]
+        q = torch.stack([t[0] for t in qkv]).contiguous()
+        k = torch.stack([t[1] for t in qkv]).contiguous()
+        v = torch.stack([t[2] for t in qkv]).contiguous()
+        del qkv
+        n_hdr = q.shape[1]
+        out = torch.empty((layers, n_hdr, g.n_q_heads, g.head_dim), dtype=torch.bfloat16, device=self.dev)
+        ws = torch.empty(run.layout.workspace_bytes(layers), dtype=torch.uint8, device=self.dev)
+        lay = run.layout
+        lay.prefill_attention(0, layers, q, k, v, out, ws, run.stream)  # untimed
+        torch.cuda.synchronize()
+        lay.profile_read()
+        lay.set_option(B.OPT_PROFILE, 1)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            lay.prefill_attention(0, layers, q, k, v, out, ws, run.stream)
+        e1.record()
+        torch.cuda.synchronize()
+        prof = lay.profile_read()
+        lay.set_option(B.OPT_PROFILE, 0)
+        run.check()
+        # keys every header row sees: instruction and context rows up to themselves, question rows the instruction,
+        # their context and their question's prefix
+        P = wl.shared_len
+        keys = P * (P + 1) // 2
+        for b in range(wl.n_prompts):
+            L = int(wl.ctx_len[b])
+            keys += L * P + L * (L + 1) // 2
+            for kq in range(int(wl.q_begin[b]), int(wl.q_begin[b + 1])):
+                n = int(wl.q_len[kq])
+                keys += n * (P + L) + n * (n + 1) // 2
+        flops = 4 * g.head_dim * g.n_q_heads * keys * layers * reps
+        att_ms = prof["attention_ms"] + prof["merge_ms"]
+        tflops = flops / (att_ms * 1e-3) / 1e12 if att_ms > 0 else 0.0
+        return {"header_tokens": int(n_hdr), "layers_per_call": layers, "calls_timed": reps,
+                "ms_per_layer_whole_call": e0.elapsed_time(e1) / (layers * reps),
+                "attention_ms_per_layer": att_ms / (layers * reps), "tflops": tflops,
+                "roofline": {"bound": "tensor", "achieved": tflops, "peak": peaks["bf16_tflops_sustained"],
+                             "unit": "TFLOP/s", "frac": tflops / peaks["bf16_tflops_sustained"],
+                             "peak_kind": peaks["kind"] + " sustained cuBLAS bf16"},
+                "api": "ippd_prefill_attention (header K/V append + attention of every header token)"}
+
     def read_probe(self, steps):
         """GB/s of the tile stream alone (the attention kernel's copies without its arithmetic) over `steps`."""
         torch = self.torch
@@ -298,7 +349,7 @@ class ConfigBench:
 
 def measure_config(name, args, dev, peaks, sync, want_layer_modes, rank_world):
     """All device-resident measurements of one configuration; returns (entry dict, ConfigBench)."""
-    cb = ConfigBench(name, dev, args.kernel)
+    cb = ConfigBench(name, dev, args.kernel, n_layers=args.layers)
     wl, g = cb.wl, cb.g
     timed = cb.prepare(spread_steps(wl.n_steps, args.steps))
     warm = cb.prepare(spread_steps(wl.n_steps, args.warmup))
@@ -346,6 +397,8 @@ def measure_config(name, args, dev, peaks, sync, want_layer_modes, rank_world):
                            min(wl.step_bytes(s)["total"] for s in range(wl.n_steps)),
                            float(np.mean([wl.step_bytes(s)["total"] for s in range(wl.n_steps)])),
                            max(wl.step_bytes(s)["total"] for s in range(wl.n_steps)))]}}
+    if want_layer_modes and args.kernel in (0, 2):
+        entry["prefill"] = cb.prefill(peaks)
     if want_layer_modes:
         modes = {}
         for lpc in (1, 4, 8):
@@ -427,7 +480,8 @@ def main():
     ap.add_argument("--kernel", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
-    ap.add_argument("--no-layer-modes", action="store_true")
+    ap.add_argument("--no-layer-modes", action="store_true", help="skip the per-layer launch modes and the prefill")
+    ap.add_argument("--layers", type=int, default=0, help="override the number of layers (profiler captures)")
     ap.add_argument("--sweep", action="store_true",
                     help="questions-per-context x context-length table (the SWEEP-L*-Q* workloads) instead of the headline line")
     args = ap.parse_args()
@@ -530,6 +584,7 @@ def main():
                                  f"{cache_mb:.0f} MB K/V cache, larger than the 126 MB L2"},
                 "roofline": entry["roofline"], "read_probe_gbs": entry["read_probe_gbs"],
                 "per_layer_mode": entry.get("per_layer_mode"), "layer_group_modes": entry.get("layer_group_modes"),
+                "prefill": entry.get("prefill"),
                 "per_config": per_config, "e2e": e2e, "cpu_baseline": cpu, "gpu_launches": int(launches),
                 "clocks": clocks, "question_tokens": tokens, "wall_s": time.perf_counter() - t_wall0}
         print(json.dumps(line), flush=True)

@@ -308,11 +308,20 @@ ippd_attn_tc_kernel(IppdDev L, IppdStepDev S, IppdTcArgs A, const __nv_bfloat16*
     while (ok && tc_next_segment(A, S, Hkv, g0, g1, g, sg)) {
       const int layer = A.layer_begin + sg.ll;
       const int seg_act_begin = S.rbs[sg.rb].act_begin, seg_n_act = S.rbs[sg.rb].n_act;
+      // the description of tile t + 1 (and its pieces) is fetched while tile t is being issued: two dependent loads
+      // from global memory that would otherwise sit between the copies of consecutive tiles
+      IppdTcTile ti = A.tiles[sg.t_begin];
+      IppdTcPiece pc;
+      pc.n_groups = 0;
+      if (lane < ti.n_pieces) pc = A.pieces[ti.piece_begin + lane];
       for (int t = sg.t_begin; t < sg.t_end && ok; ++t, ++tc) {
-        const IppdTcTile ti = A.tiles[t];
-        IppdTcPiece pc;
-        pc.n_groups = 0;
-        if (lane < ti.n_pieces) pc = A.pieces[ti.piece_begin + lane];
+        IppdTcTile ti_next = ti;
+        IppdTcPiece pc_next;
+        pc_next.n_groups = 0;
+        if (t + 1 < sg.t_end) {
+          ti_next = A.tiles[t + 1];
+          if (lane < ti_next.n_pieces) pc_next = A.pieces[ti_next.piece_begin + lane];
+        }
         TcMeta& mt = sh->meta[tc % IPPD_TC_NMETA];
         if (lane == 0) { mt.rows = ti.rows; mt.n_pieces = ti.n_pieces; }
         if (ti.n_pieces > 0) {
@@ -371,6 +380,8 @@ ippd_attn_tc_kernel(IppdDev L, IppdStepDev S, IppdTcArgs A, const __nv_bfloat16*
                      (uint32_t)pc.n_groups * GB, &sh->kv_full[buf]);
           }
         }
+        ti = ti_next;
+        pc = pc_next;
       }
     }
     if (lane == 0) {
