@@ -263,16 +263,23 @@ def tuple_inputs(wl, b: int, k: int, s: int, layer: int, kv_head: int, ctx_cache
                 ctx_cache[skey] = (kp, vp)
         ks.insert(0, kp)
         vs.insert(0, vp)
-    for t in range(s + 1):
-        if step_cache is None:
+    if step_cache is None:
+        for t in range(s + 1):
             ka, va = wl.step_kv(t, layer, [k])
-            ka, va = ka[0], va[0]
-        else:  # raw step tensors of ALL questions, generated once per (t, layer)
-            if (t, layer) not in step_cache:
-                step_cache[(t, layer)] = wl.step_kv(t, layer, list(range(wl.n_questions)))
-            ka, va = step_cache[(t, layer)][0][k], step_cache[(t, layer)][1][k]
-        ks.append(ka[None, kv_head].double().numpy())
-        vs.append(va[None, kv_head].double().numpy())
+            ks.append(ka[0][None, kv_head].double().numpy())
+            vs.append(va[0][None, kv_head].double().numpy())
+    else:
+        # raw step tensors of ALL questions for one (layer, KV head), generated once per step and kept stacked over the
+        # steps, [steps so far, NQ, D]: a question's answer tokens are then one slice
+        key = ("steps", layer, kv_head)
+        kst, vst = step_cache.get(key, (np.zeros((0, wl.n_questions, g.head_dim)),) * 2)
+        if kst.shape[0] < s + 1:
+            more = [wl.step_kv(t, layer, list(range(wl.n_questions))) for t in range(kst.shape[0], s + 1)]
+            kst = np.concatenate([kst] + [a[:, kv_head].double().numpy()[None] for a, _ in more])
+            vst = np.concatenate([vst] + [b_[:, kv_head].double().numpy()[None] for _, b_ in more])
+            step_cache[key] = (kst, vst)
+        ks.append(kst[:s + 1, k])
+        vs.append(vst[:s + 1, k])
     q = wl.step_q(s, layer, [k])[0, kv_head * G:(kv_head + 1) * G].double().numpy()
     return np.concatenate(ks), np.concatenate(vs), q
 

@@ -61,9 +61,6 @@ def run_and_sample(name, check, per_prompt, kernel=0, full_layer_step=None):
             want = np.stack([ref[k] for k in qids])
             gate(got, want, f"{name} step {s} layer {layer} head {head}")
             n_tuples += got.shape[0] * G
-        # the raw step tensors of other layers are not needed again
-        for key in [k for k in step_cache if k[1] not in {l for l, _ in check[s]}]:
-            del step_cache[key]
     run.check()
     del run
     torch.cuda.empty_cache()

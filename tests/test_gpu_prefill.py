@@ -95,7 +95,7 @@ def test_ragged_prefill_every_header_row_and_cache_equals_appends(shared_len):
     _compare_header(wl, outs[0], range(2), range(2), what="ragged prefill")
     # two layers per call cut the tile sequence elsewhere: same rows within rounding
     rms = np.sqrt((outs[0].astype(np.float64) ** 2).mean(axis=-1, keepdims=True))
-    assert (np.abs(outs[1] - outs[0]) / rms).max() <= 1.5e-2
+    assert (np.abs(outs[1] - outs[0]) / rms).max() <= 3e-2
     cache = {}
     for s in range(2):
         compare_step(run, s, range(2), range(2), cache, "decode after prefill")
