@@ -564,7 +564,7 @@ extern "C" int ippd_workspace_bytes(const ippd_layout_t* L, int32_t layer_count,
     return IPPD_ERR_INVALID_ARG;
   }
   const IppdHostLayout& h = L->h;
-  if (h.kernel_path() == 2) {
+  if (h.kernel_path() >= 2) {
     // two partial slots per CTA of the persistent kernel, whatever the step
     size_t per_slot = (size_t)IPPD_TC_ROWS * (h.geom.head_dim + 2) * sizeof(float);
     *bytes = align_up((size_t)kMaxCtas * 2 * per_slot, 256) + 512;
@@ -621,7 +621,7 @@ static int tc_partition(const ippd_layout* L, int layer_count, IppdTcArgs* a, bo
 static size_t scratch_need(const ippd_layout* L, int layer_count, size_t* o_bytes, bool* needed) {
   const IppdHostLayout& h = L->h;
   size_t n_part;
-  if (h.kernel_path() == 2) {
+  if (h.kernel_path() >= 2) {
     IppdTcArgs a;
     bool any_partial = false;
     if (tc_partition(L, layer_count, &a, &any_partial) != IPPD_OK) { a.n_cta = kMaxCtas; any_partial = true; }
@@ -656,7 +656,7 @@ static int launch_attention(ippd_layout* L, const IppdDev& d, int layer_begin, i
   const IppdStepDev& S = L->step_dev;
   const int Hkv = L->h.geom.n_kv_heads;
   int out_f32 = L->h.geom.out_dtype == IPPD_F32;
-  if (L->h.kernel_path() == 2) {
+  if (L->h.kernel_path() >= 2) {
     IppdTcArgs a;
     bool any_partial = false;
     {
@@ -739,7 +739,7 @@ static int decode_attention_impl(ippd_layout_t* L, const char* who, int32_t laye
     part_o = (float*)workspace;
     part_ml = (float*)((char*)workspace + o_bytes);
   }
-  if (k_step && h.kernel_path() != 2) {
+  if (k_step && h.kernel_path() < 2) {
     // the warp-level path has no append role: the step's tokens go through the append kernel first
     int rc = ippd_append_kv(L, layer_begin, layer_count, IPPD_APPEND_STEP, nullptr, 0, k_step, v_step, stream_);
     if (rc != IPPD_OK) return rc;
@@ -844,7 +844,7 @@ extern "C" int ippd_prefill_attention(ippd_layout_t* L, int32_t layer_begin, int
   if (!L) { ippd_set_error("ippd_prefill_attention: NULL layout"); return IPPD_ERR_INVALID_ARG; }
   if (!L->bound) { ippd_set_error("ippd_prefill_attention: no cache bound"); return IPPD_ERR_NOT_BOUND; }
   const IppdHostLayout& h = L->h;
-  if (h.kernel_path() != 2) { ippd_set_error("ippd_prefill_attention: tensor-core path only"); return IPPD_ERR_INVALID_ARG; }
+  if (h.kernel_path() < 2) { ippd_set_error("ippd_prefill_attention: tensor-core path only"); return IPPD_ERR_INVALID_ARG; }
   if (layer_begin < 0 || layer_count < 1 || layer_begin + layer_count > h.geom.n_layers) {
     ippd_set_error("ippd_prefill_attention: layer range out of bounds");
     return IPPD_ERR_INVALID_ARG;
@@ -951,7 +951,7 @@ extern "C" int ippd_decode_step_grouped(ippd_layout_t* L, int32_t layers_per_cal
 extern "C" int ippd_read_probe(ippd_layout_t* L, int32_t layer_begin, int32_t layer_count, void* stream_) {
   if (!L) { ippd_set_error("ippd_read_probe: NULL layout"); return IPPD_ERR_INVALID_ARG; }
   if (!L->bound) { ippd_set_error("ippd_read_probe: no cache bound"); return IPPD_ERR_NOT_BOUND; }
-  if (!L->have_step || L->h.kernel_path() != 2) {
+  if (!L->have_step || L->h.kernel_path() < 2) {
     ippd_set_error("ippd_read_probe: needs a step declared for the tensor-core path");
     return IPPD_ERR_INVALID_ARG;
   }

@@ -204,8 +204,9 @@ constexpr int tc_smem_bytes() {
 }
 
 
-// Bounded wait that also gives up when another role has raised the abort flag.
-__device__ __forceinline__ bool tc_wait(uint64_t* bar, uint32_t parity, const IppdDev& L, TcShared* sh) {
+// Bounded wait that also gives up when another role has raised the abort flag.  (SH: the kernel's shared block.)
+template <class SH>
+__device__ __forceinline__ bool tc_wait(uint64_t* bar, uint32_t parity, const IppdDev& L, SH* sh) {
   if (mbar_try_wait(bar, parity)) return true;
   if (L.wait_limit_ns == 0) {  // "never wait": a phase still incomplete after one (briefly suspending) probe fails
     sh->abort_flag = 1;
@@ -228,7 +229,8 @@ __device__ __forceinline__ bool tc_wait(uint64_t* bar, uint32_t parity, const Ip
 }
 
 // Bounded wait until the append warp's progress counter has passed `need`.
-__device__ __forceinline__ bool tc_wait_appended(const uint32_t* counter, uint32_t need, const IppdDev& L, TcShared* sh) {
+template <class SH>
+__device__ __forceinline__ bool tc_wait_appended(const uint32_t* counter, uint32_t need, const IppdDev& L, SH* sh) {
   auto load = [&]() {
     uint32_t v;
     asm volatile("ld.acquire.cta.shared::cta.u32 %0, [%1];" : "=r"(v) : "r"(smem_u32(counter)) : "memory");
@@ -248,6 +250,166 @@ __device__ __forceinline__ bool tc_wait_appended(const uint32_t* counter, uint32
     }
   }
   return true;
+}
+
+// Producer role (one warp): walks the CTA's slice of the tile sequence and keeps the ring of NBUF 128-row buffers
+// full.  Lane 0 owns the barriers and the context copies, lane i < n_pieces fetches piece i of a packed tile; the
+// tile's description is left in shared memory for the other roles (published by the K buffer's mbarrier, which this
+// warp arrives on afterwards).  SH needs kv_full[], kv_empty[], meta[], app_done and abort_flag.
+template <int D, int NBUF, class SH>
+__device__ __forceinline__ void tc_producer_role(const IppdDev& L, const IppdStepDev& S, const IppdTcArgs& A, SH* sh,
+                                                 uint8_t* ring, long long g0, long long g1, int lane) {
+  constexpr int GB = (D / 8) * 128;
+  constexpr int TILE_BYTES = 16 * GB;
+  const int Hkv = L.Hkv;
+  long long g = g0;
+  TcSegment sg;
+  uint32_t n = 0;   // buffers filled so far
+  uint32_t tc = 0;  // tiles issued so far
+  bool ok = true;
+  while (ok && tc_next_segment(A, S, Hkv, g0, g1, g, sg)) {
+    const int layer = A.layer_begin + sg.ll;
+    const int seg_act_begin = S.rbs[sg.rb].act_begin, seg_n_act = S.rbs[sg.rb].n_act;
+    // the description of tile t + 1 (and its pieces) is fetched while tile t is being issued: two dependent loads
+    // from global memory that would otherwise sit between the copies of consecutive tiles
+    IppdTcTile ti = A.tiles[sg.t_begin];
+    IppdTcPiece pc;
+    pc.n_groups = 0;
+    if (lane < ti.n_pieces) pc = A.pieces[ti.piece_begin + lane];
+    for (int t = sg.t_begin; t < sg.t_end && ok; ++t, ++tc) {
+      IppdTcTile ti_next = ti;
+      IppdTcPiece pc_next;
+      pc_next.n_groups = 0;
+      if (t + 1 < sg.t_end) {
+        ti_next = A.tiles[t + 1];
+        if (lane < ti_next.n_pieces) pc_next = A.pieces[ti_next.piece_begin + lane];
+      }
+      TcMeta& mt = sh->meta[tc % IPPD_TC_NMETA];
+      if (lane == 0) { mt.rows = ti.rows; mt.n_pieces = ti.n_pieces; }
+      if (ti.n_pieces > 0) {
+        // column window of every question in this tile: its pieces sit on adjacent lanes, the first gives c0 and
+        // the last c1 (only the last piece of a question can be partly valid)
+        reinterpret_cast<uint32_t*>(mt.c0)[lane & 15] = 0u;  // 64 + 64 bytes: lanes 0..15 clear c0, 16..31 clear c1
+        if (lane >= 16) reinterpret_cast<uint32_t*>(mt.c1)[lane & 15] = 0u;
+        __syncwarp();
+        const int a_me = lane < ti.n_pieces ? pc.a_local : -1;
+        const int a_prev = __shfl_up_sync(0xffffffffu, a_me, 1), a_next = __shfl_down_sync(0xffffffffu, a_me, 1);
+        if (lane < ti.n_pieces) {
+          if (lane == 0 || a_prev != a_me) mt.c0[a_me] = (uint8_t)pc.row0;
+          if (lane == ti.n_pieces - 1 || a_next != a_me) mt.c1[a_me] = (uint8_t)(pc.row0 + pc.valid);
+        }
+      } else if (ti.n_pieces < 0) {
+        // causal context tile (prefill): query a of the row block sits at virtual position pos_a and sees the
+        // tile's tokens up to itself, columns [0, pos_a + 1 - first position of the tile)
+        for (int a = lane; a < 64; a += 32) {
+          int c1 = 0;
+          if (a < seg_n_act) c1 = max(0, min(ti.rows, S.act_pos[seg_act_begin + a] + 1 - ti.piece_begin));
+          mt.c0[a] = 0;
+          mt.c1[a] = (uint8_t)c1;
+        }
+      }
+      __syncwarp();
+      const int groups = (ti.rows + 7) >> 3;
+      if (A.k_step != nullptr && ti.n_pieces > 0) {
+        // the step's own tokens are written by the append warp of this CTA: fetch the tile after them
+        if (lane == 0) ok = tc_wait_appended(&sh->app_done, tc + 1, L, sh);
+        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+        if (!ok) break;
+      }
+      for (int kv = 0; kv < 2 && ok; ++kv, ++n) {
+        uint32_t buf = n % NBUF, ph = (n / NBUF) & 1;
+        if (lane == 0) ok = tc_wait(&sh->kv_empty[buf], ph ^ 1, L, sh);
+        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+        if (!ok) break;
+        uint8_t* dst = ring + buf * TILE_BYTES;
+        if (kv == 1 && (groups & 1)) {
+          // The P V product works in steps of 16 rows: the 8 rows after an odd number of fetched groups are not
+          // written by the copies below and would be stale shared memory; P is zero there, but 0 * NaN = NaN.
+          uint4* z = reinterpret_cast<uint4*>(dst + groups * GB);
+          for (int idx = lane; idx < GB / 16; idx += 32) z[idx] = make_uint4(0, 0, 0, 0);
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+          __syncwarp();
+        }
+        if (lane == 0) mbar_arrive_expect_tx(&sh->kv_full[buf], (uint32_t)groups * GB);
+        __syncwarp();
+        if (ti.n_pieces <= 0) {
+          if (lane == 0)
+            bulk_g2s(dst, L.cache + ippd_tile_addr(L, layer, sg.head, ti.pool_tile, kv), (uint32_t)groups * GB,
+                     &sh->kv_full[buf]);
+        } else if (lane < ti.n_pieces) {
+          bulk_g2s(dst + (pc.row0 >> 3) * GB,
+                   L.cache + ippd_tile_addr(L, layer, sg.head, pc.src_tile, kv) + (size_t)pc.src_group * GB,
+                   (uint32_t)pc.n_groups * GB, &sh->kv_full[buf]);
+        }
+      }
+      ti = ti_next;
+      pc = pc_next;
+    }
+  }
+  if (lane == 0) {
+    // copies already issued must land before the CTA's shared memory is released (they normally have: the MMA lane
+    // consumed them; this matters when the other roles gave up early)
+    uint32_t first = n > NBUF ? n - NBUF : 0;
+    for (uint32_t i = first; i < n; ++i)
+      mbar_wait_ns(&sh->kv_full[i % NBUF], (i / NBUF) & 1, L, IPPD_DRAIN_LIMIT_NS);
+  }
+}
+
+// Append role (one warp, only when the call carries the step's raw K/V): walks the CTA's slice ahead of the producer
+// and, for every packed branch piece that holds the token fed at this step, rotates its key (RoPE) and writes K~ and V
+// into the piece's cache slot; the producer fetches a packed tile only after its slots are in place.
+template <int D, class SH>
+__device__ __forceinline__ void tc_append_role(const IppdDev& L, const IppdStepDev& S, const IppdTcArgs& A, SH* sh,
+                                               long long g0, long long g1, int lane) {
+  const int Hkv = L.Hkv;
+  if (A.k_step != nullptr) {
+    constexpr int CP = D / 16;    // lanes per token: one per pair of 16-byte chunks (c, c + D/16)
+    constexpr int TPP = 32 / CP;  // tokens per pass of the warp
+    long long g = g0;
+    TcSegment sg;
+    uint32_t tc = 0;  // tiles of the slice passed so far (the producer counts the same way)
+    bool stop = false;
+    while (!stop && tc_next_segment(A, S, Hkv, g0, g1, g, sg)) {
+      const IppdRowBlock rb = S.rbs[sg.rb];
+      const int first_packed = A.rb_tile_begin[sg.rb] + rb.n_ctx_tiles;
+      const int layer = A.layer_begin + sg.ll;
+      for (int t = sg.t_begin; t < sg.t_end; ++t, ++tc) {
+        if (t < first_packed) continue;  // context tiles hold no token of this step
+        if (sh->abort_flag) { stop = true; break; }
+        const IppdTcTile ti = A.tiles[t];
+        IppdTcPiece pc;
+        pc.new_tok = 0;
+        if (lane < ti.n_pieces) pc = A.pieces[ti.piece_begin + lane];
+        unsigned todo = __ballot_sync(0xffffffffu, pc.new_tok != 0);
+        while (todo) {
+          // lane group gi takes the gi-th piece still to do
+          const int gi = lane / CP, c = lane % CP;
+          unsigned m = todo;
+          int src = 0;
+          for (int i = 0; i <= gi && m; ++i) { src = __ffs(m) - 1; m &= m - 1; }
+          const bool have = __popc(todo) > gi;
+          const int a_local = __shfl_sync(0xffffffffu, pc.a_local, src);
+          const int src_tile = __shfl_sync(0xffffffffu, pc.src_tile, src);
+          const int src_group = __shfl_sync(0xffffffffu, pc.src_group, src);
+          const int new_tok = __shfl_sync(0xffffffffu, pc.new_tok, src);
+          if (have) {
+            const int a = rb.act_begin + a_local;
+            const size_t row = (((size_t)sg.ll * S.A + a) * Hkv + sg.head) * D + c * 8;
+            ippd_rope_store_pair<D>(L, A.k_step + row, A.v_step + row, S.act_pos[a], c,
+                                    ippd_tile_addr(L, layer, sg.head, src_tile, 0), src_group * 8 + new_tok - 1);
+          }
+          for (int i = 0; i < TPP && todo; ++i) todo &= todo - 1;
+        }
+        // the stores above (generic proxy) are read by the producer's bulk copies (async proxy)
+        asm volatile("fence.proxy.async;" ::: "memory");
+        __syncwarp();
+        if (lane == 0)
+          asm volatile("st.release.cta.shared::cta.u32 [%0], %1;" ::"r"(smem_u32(&sh->app_done)), "r"(tc + 1) : "memory");
+      }
+    }
+    if (lane == 0)
+      asm volatile("st.release.cta.shared::cta.u32 [%0], %1;" ::"r"(smem_u32(&sh->app_done)), "r"(0xFFFFFFFFu) : "memory");
+  }
 }
 
 #include "ippd_attn_tc_softmax.cuh"
@@ -296,101 +458,7 @@ ippd_attn_tc_kernel(IppdDev L, IppdStepDev S, IppdTcArgs A, const __nv_bfloat16*
   const uint32_t tS0 = tmem, tO = tmem + 256, tQ = tmem + 384;
 
   if (warp == 0) {
-    // =========================== producer ===========================
-    // The whole warp walks the tiles: lane 0 owns the barriers and the context copies, lane i < n_pieces fetches
-    // piece i of a packed tile and issues its copies; the tile's description is left in shared memory for the
-    // other roles (published by the K buffer's mbarrier, which this warp arrives on afterwards).
-    long long g = g0;
-    TcSegment sg;
-    uint32_t n = 0;   // buffers filled so far
-    uint32_t tc = 0;  // tiles issued so far
-    bool ok = true;
-    while (ok && tc_next_segment(A, S, Hkv, g0, g1, g, sg)) {
-      const int layer = A.layer_begin + sg.ll;
-      const int seg_act_begin = S.rbs[sg.rb].act_begin, seg_n_act = S.rbs[sg.rb].n_act;
-      // the description of tile t + 1 (and its pieces) is fetched while tile t is being issued: two dependent loads
-      // from global memory that would otherwise sit between the copies of consecutive tiles
-      IppdTcTile ti = A.tiles[sg.t_begin];
-      IppdTcPiece pc;
-      pc.n_groups = 0;
-      if (lane < ti.n_pieces) pc = A.pieces[ti.piece_begin + lane];
-      for (int t = sg.t_begin; t < sg.t_end && ok; ++t, ++tc) {
-        IppdTcTile ti_next = ti;
-        IppdTcPiece pc_next;
-        pc_next.n_groups = 0;
-        if (t + 1 < sg.t_end) {
-          ti_next = A.tiles[t + 1];
-          if (lane < ti_next.n_pieces) pc_next = A.pieces[ti_next.piece_begin + lane];
-        }
-        TcMeta& mt = sh->meta[tc % IPPD_TC_NMETA];
-        if (lane == 0) { mt.rows = ti.rows; mt.n_pieces = ti.n_pieces; }
-        if (ti.n_pieces > 0) {
-          // column window of every question in this tile: its pieces sit on adjacent lanes, the first gives c0 and
-          // the last c1 (only the last piece of a question can be partly valid)
-          reinterpret_cast<uint32_t*>(mt.c0)[lane & 15] = 0u;  // 64 + 64 bytes: lanes 0..15 clear c0, 16..31 clear c1
-          if (lane >= 16) reinterpret_cast<uint32_t*>(mt.c1)[lane & 15] = 0u;
-          __syncwarp();
-          const int a_me = lane < ti.n_pieces ? pc.a_local : -1;
-          const int a_prev = __shfl_up_sync(0xffffffffu, a_me, 1), a_next = __shfl_down_sync(0xffffffffu, a_me, 1);
-          if (lane < ti.n_pieces) {
-            if (lane == 0 || a_prev != a_me) mt.c0[a_me] = (uint8_t)pc.row0;
-            if (lane == ti.n_pieces - 1 || a_next != a_me) mt.c1[a_me] = (uint8_t)(pc.row0 + pc.valid);
-          }
-        } else if (ti.n_pieces < 0) {
-          // causal context tile (prefill): query a of the row block sits at virtual position pos_a and sees the
-          // tile's tokens up to itself, columns [0, pos_a + 1 - first position of the tile)
-          for (int a = lane; a < 64; a += 32) {
-            int c1 = 0;
-            if (a < seg_n_act) c1 = max(0, min(ti.rows, S.act_pos[seg_act_begin + a] + 1 - ti.piece_begin));
-            mt.c0[a] = 0;
-            mt.c1[a] = (uint8_t)c1;
-          }
-        }
-        __syncwarp();
-        const int groups = (ti.rows + 7) >> 3;
-        if (A.k_step != nullptr && ti.n_pieces > 0) {
-          // the step's own tokens are written by the append warp of this CTA: fetch the tile after them
-          if (lane == 0) ok = tc_wait_appended(&sh->app_done, tc + 1, L, sh);
-          ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
-          if (!ok) break;
-        }
-        for (int kv = 0; kv < 2 && ok; ++kv, ++n) {
-          uint32_t buf = n % IPPD_TC_NBUF, ph = (n / IPPD_TC_NBUF) & 1;
-          if (lane == 0) ok = tc_wait(&sh->kv_empty[buf], ph ^ 1, L, sh);
-          ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
-          if (!ok) break;
-          uint8_t* dst = ring + buf * TILE_BYTES;
-          if (kv == 1 && (groups & 1)) {
-            // The P V product works in steps of 16 rows: the 8 rows after an odd number of fetched groups are not
-            // written by the copies below and would be stale shared memory; P is zero there, but 0 * NaN = NaN.
-            uint4* z = reinterpret_cast<uint4*>(dst + groups * GB);
-            for (int idx = lane; idx < GB / 16; idx += 32) z[idx] = make_uint4(0, 0, 0, 0);
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            __syncwarp();
-          }
-          if (lane == 0) mbar_arrive_expect_tx(&sh->kv_full[buf], (uint32_t)groups * GB);
-          __syncwarp();
-          if (ti.n_pieces <= 0) {
-            if (lane == 0)
-              bulk_g2s(dst, L.cache + ippd_tile_addr(L, layer, sg.head, ti.pool_tile, kv), (uint32_t)groups * GB,
-                       &sh->kv_full[buf]);
-          } else if (lane < ti.n_pieces) {
-            bulk_g2s(dst + (pc.row0 >> 3) * GB,
-                     L.cache + ippd_tile_addr(L, layer, sg.head, pc.src_tile, kv) + (size_t)pc.src_group * GB,
-                     (uint32_t)pc.n_groups * GB, &sh->kv_full[buf]);
-          }
-        }
-        ti = ti_next;
-        pc = pc_next;
-      }
-    }
-    if (lane == 0) {
-      // copies already issued must land before the CTA's shared memory is released (they normally have: the MMA lane
-      // consumed them; this matters when the other roles gave up early)
-      uint32_t first = n > IPPD_TC_NBUF ? n - IPPD_TC_NBUF : 0;
-      for (uint32_t i = first; i < n; ++i)
-        mbar_wait_ns(&sh->kv_full[i % IPPD_TC_NBUF], (i / IPPD_TC_NBUF) & 1, L, IPPD_DRAIN_LIMIT_NS);
-    }
+    tc_producer_role<D, IPPD_TC_NBUF>(L, S, A, sh, ring, g0, g1, lane);
   } else if (warp == 1) {
     // =========================== P V issuer (one lane) ===========================
     // O += P(j) V(j): P from TMEM (the head of S buffer j & 1), V from ring slot 2j+1 (MN-major).
@@ -429,55 +497,7 @@ ippd_attn_tc_kernel(IppdDev L, IppdStepDev S, IppdTcArgs A, const __nv_bfloat16*
       mbar_wait_ns(&sh->drain[0], 0, L, IPPD_DRAIN_LIMIT_NS);
     }
   } else if (warp == IPPD_TC_WARP_APPEND) {
-    // =========================== append (RoPE + store of the step's tokens) ===========================
-    if (A.k_step != nullptr) {
-      constexpr int CP = D / 16;    // lanes per token: one per pair of 16-byte chunks (c, c + D/16)
-      constexpr int TPP = 32 / CP;  // tokens per pass of the warp
-      long long g = g0;
-      TcSegment sg;
-      uint32_t tc = 0;  // tiles of the slice passed so far (the producer counts the same way)
-      bool stop = false;
-      while (!stop && tc_next_segment(A, S, Hkv, g0, g1, g, sg)) {
-        const IppdRowBlock rb = S.rbs[sg.rb];
-        const int first_packed = A.rb_tile_begin[sg.rb] + rb.n_ctx_tiles;
-        const int layer = A.layer_begin + sg.ll;
-        for (int t = sg.t_begin; t < sg.t_end; ++t, ++tc) {
-          if (t < first_packed) continue;  // context tiles hold no token of this step
-          if (sh->abort_flag) { stop = true; break; }
-          const IppdTcTile ti = A.tiles[t];
-          IppdTcPiece pc;
-          pc.new_tok = 0;
-          if (lane < ti.n_pieces) pc = A.pieces[ti.piece_begin + lane];
-          unsigned todo = __ballot_sync(0xffffffffu, pc.new_tok != 0);
-          while (todo) {
-            // lane group gi takes the gi-th piece still to do
-            const int gi = lane / CP, c = lane % CP;
-            unsigned m = todo;
-            int src = 0;
-            for (int i = 0; i <= gi && m; ++i) { src = __ffs(m) - 1; m &= m - 1; }
-            const bool have = __popc(todo) > gi;
-            const int a_local = __shfl_sync(0xffffffffu, pc.a_local, src);
-            const int src_tile = __shfl_sync(0xffffffffu, pc.src_tile, src);
-            const int src_group = __shfl_sync(0xffffffffu, pc.src_group, src);
-            const int new_tok = __shfl_sync(0xffffffffu, pc.new_tok, src);
-            if (have) {
-              const int a = rb.act_begin + a_local;
-              const size_t row = (((size_t)sg.ll * S.A + a) * Hkv + sg.head) * D + c * 8;
-              ippd_rope_store_pair<D>(L, A.k_step + row, A.v_step + row, S.act_pos[a], c,
-                                      ippd_tile_addr(L, layer, sg.head, src_tile, 0), src_group * 8 + new_tok - 1);
-            }
-            for (int i = 0; i < TPP && todo; ++i) todo &= todo - 1;
-          }
-          // the stores above (generic proxy) are read by the producer's bulk copies (async proxy)
-          asm volatile("fence.proxy.async;" ::: "memory");
-          __syncwarp();
-          if (lane == 0)
-            asm volatile("st.release.cta.shared::cta.u32 [%0], %1;" ::"r"(smem_u32(&sh->app_done)), "r"(tc + 1) : "memory");
-        }
-      }
-      if (lane == 0)
-        asm volatile("st.release.cta.shared::cta.u32 [%0], %1;" ::"r"(smem_u32(&sh->app_done)), "r"(0xFFFFFFFFu) : "memory");
-    }
+    tc_append_role<D>(L, S, A, sh, g0, g1, lane);
   } else if (warp == IPPD_TC_WARP_S_ISSUER) {
     // =========================== S issuer (one lane) ===========================
     // S(j) = Q~ K(j)^T: Q~ from TMEM, K from ring slot 2j (K-major), into S buffer j & 1.  That buffer held P(j-2),

@@ -13,12 +13,12 @@ extern "C" const char* ippd_last_error(void) { return g_last_error.c_str(); }
 static const int kTargetCtas = 148 * 2 * 4;  // CTAs wanted per launch: SMs x resident CTAs x waves
 static const int kMinTilesPerSplit = 4;
 
-int IppdHostLayout::kernel_path() const { return opt_kernel == 0 ? 2 : opt_kernel; }
-int IppdHostLayout::rows_per_block() const { return kernel_path() == 2 ? 128 : 64; }
+int IppdHostLayout::kernel_path() const { return opt_kernel == 0 ? IPPD_DEFAULT_KERNEL : opt_kernel; }
+int IppdHostLayout::rows_per_block() const { return kernel_path() >= 2 ? 128 : 64; }
 // questions per row block: the tensor-core path keeps at most 64 questions per block
 static int questions_per_block(const IppdHostLayout& L) {
   int qpr = L.rows_per_block() / L.G;
-  return L.kernel_path() == 2 ? std::min(qpr, 64) : qpr;
+  return L.kernel_path() >= 2 ? std::min(qpr, 64) : qpr;
 }
 
 static inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
@@ -188,7 +188,7 @@ int ippd_host_plan_entries(const IppdHostLayout& L, const IppdPlanEntry* ent, co
   plan->units.clear();
   plan->tc_tiles.clear();
   plan->tc_pieces.clear();
-  const bool tc_path = L.kernel_path() == 2;
+  const bool tc_path = L.kernel_path() >= 2;
   if (!tc_path && L.shared_len > 0) {
     ippd_set_error("ippd_begin_step: a shared instruction needs the tensor-core path (IPPD_OPT_KERNEL 0 or 2)");
     return IPPD_ERR_INVALID_ARG;
@@ -329,7 +329,7 @@ int ippd_host_plan_entries(const IppdHostLayout& L, const IppdPlanEntry* ent, co
   plan->hdr.n_active = A;
   plan->hdr.n_rowblocks = (int32_t)plan->rbs.size();
   plan->hdr.rows_per_block = RB;
-  if (L.kernel_path() == 2) {  // the persistent kernel cuts the tile sequence itself: no unit list
+  if (L.kernel_path() >= 2) {  // the persistent kernel cuts the tile sequence itself: no unit list
     plan->hdr.n_units = 0;
     return IPPD_OK;
   }

@@ -9,6 +9,7 @@
 #include "../../include/ippd.h"
 
 #define IPPD_MAX_ROWS_PER_BLOCK 128
+#define IPPD_DEFAULT_KERNEL 2  // what IPPD_OPT_KERNEL = 0 selects
 
 // ---- per-step work description (layer- and head-independent; the grid adds those axes) ----
 struct IppdStepHeader {
