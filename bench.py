@@ -33,9 +33,11 @@ METRIC = "IPPD decode-attn question-tokens/s"
 UNIT = "question-tokens/s"
 HEADLINE = "C4"
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per algorithmic byte of the attention kernel, from ncu
-# captures of one launch each (summaries under profiles/: tcgen05_path_<config>_attn_*.md); the traffic of an average
-# launch is that ratio times its algorithmic bytes (traffic grows in proportion to the bytes streamed)
-NCU_TRAFFIC_RATIO = {"C2": (372.05 + 9.98) / 370.54}
+# captures of two launches each (summaries under profiles/: tcgen05_path_C2_attn_full_set.md and
+# tcgen05_path_dram_traffic_C3_C4_C5_S3.md; C4 and S3 captured with fewer layers, traffic per launch grows in proportion
+# to the layers); the traffic of an average launch is that ratio times its algorithmic bytes.  C5's ratio depends on
+# how many 128-row blocks a prompt still has (2.5 .. 4.8 over its schedule): no single figure, reported as null.
+NCU_TRAFFIC_RATIO = {"C2": 1.040, "C3": 1.009, "C4": 1.238, "S3": 2.031}
 
 
 def load_peaks():
