@@ -410,9 +410,14 @@ def measure_config(name, args, dev, peaks, sync, want_layer_modes, rank_world):
             n0 = cb.run.layout.launch_count()
             m = cb.timed(warm[:3], timed, sync)
             n1 = cb.run.layout.launch_count()
+            pm = cb.profile(timed[: max(1, 16 // max(1, g.n_layers // lpc)) + 1])  # every launch bracketed
+            calls = max(1, pm["n_attention"])
             modes[str(lpc)] = {"layers_per_call": lpc, "ms_per_step": m / len(timed),
                                "value": rank_world * tokens / (m * 1e-3),
-                               "launches_per_step": (n1 - n0) / (len(timed) + 3)}
+                               "launches_per_step": (n1 - n0) / (len(timed) + 3),
+                               "us_per_call": 1e3 * m / len(timed) / -(-g.n_layers // lpc),
+                               "bracketed_attention_us_per_call": 1e3 * pm["attention_ms"] / calls,
+                               "bracketed_merge_us_per_call": 1e3 * pm["merge_ms"] / calls}
         cb.run.set_layers_per_call(g.n_layers)
         entry["per_layer_mode"] = modes.get("1")
         entry["layer_group_modes"] = modes
