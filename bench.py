@@ -10,7 +10,7 @@ the K timed steps are spread evenly over the whole schedule instead of being its
   python bench.py [--gpus N] [--steps K] [--warmup W] [--config C4] [--also C2,C3,C5] [--impl ours|reference]
 
 Prints ONE JSON line.  The headline workload is C4 (the largest Llama-3-8B-geometry configuration that fits one GPU);
-`per_config` carries the same measurements for the other configurations.  With N > 1 (launched by torchrun) every rank
+`per_config` carries the same measurements for the other configurations (C2, C3, C5 and the second family S1, S2, S3).  With N > 1 (launched by torchrun) every rank
 runs an independent replica of the workload on its own GPU: the path is never sharded, there is no data-path
 collective.
 """
@@ -520,7 +520,8 @@ def main():
     peaks = load_peaks()
     also = args.also
     if also is None:
-        also = ",".join(c for c in ("C2", "C3", "C5") if c != args.config) if (args.config == HEADLINE and world == 1) else ""
+        also = ",".join(c for c in ("C2", "C3", "C5", "S1", "S2", "S3") if c != args.config) \
+            if (args.config == HEADLINE and world == 1) else ""
     others = [c for c in also.split(",") if c]
 
     def sync_all():
