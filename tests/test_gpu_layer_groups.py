@@ -37,3 +37,25 @@ def test_more_than_64_active_questions(kernel):
     cache = {}
     for s in range(wl.n_steps):
         compare_step(run, s, [0], range(geom.n_kv_heads), cache, "many questions")
+
+
+def test_read_probe_streams_the_step_and_changes_nothing():
+    # the measuring aid walks the same tile list as the attention kernel and discards it: no output, no error, the
+    # cache untouched, and the step it was declared for still computes correctly afterwards
+    import torch
+    geom = W.Geometry(2, 8, 2, 128, 5e5)
+    wl = W.custom_workload("probe", geom, 43, [700, 130], [5, 40], [20] * 45, [3] * 45)
+    run = PoisonedRunner(wl, out_dtype=B.F32)
+    run.load_header()
+    run.run_step(0)
+    snapshot = run.cache.clone()
+    act = wl.active(1)
+    run.layout.begin_step(act, np.full(len(act), 1, dtype=np.int32), run.stream)
+    for _ in range(3):
+        run.layout.read_probe(0, geom.n_layers, run.stream)
+    run.check()
+    assert torch.equal(snapshot, run.cache)
+    t = run.layout.host_time_read()
+    assert t["steps"] >= 1 and t["begin_step_us"] > 0
+    cache = {}
+    compare_step(run, 1, range(2), range(2), cache, "after the probe")
