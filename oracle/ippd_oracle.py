@@ -31,6 +31,12 @@ What is defined here (paper sections in brackets):
   Pinned by: the dense formulation over a stacked sequence assembled independently
   in the tests, with the KV head of each query head chosen by an explicit repeat.
 
+* `quantize_e4m3`      -- the 8-bit cache variant (not in the paper: a storage format of this build): the
+  rotated key and the value are kept as e4m3 numbers (1 sign, 4 exponent bits with bias 7, 3 mantissa bits,
+  subnormals, largest magnitude 448, no infinity), rounded to nearest-even and saturating; `standalone_attend(...,
+  kv_e4m3=True)` and `attend_tuple(..., kv_e4m3=True)` evaluate the same definition over the quantised keys and
+  values.  Pinned by: the enumeration of all 254 finite codes, hand values, and the library's float8 cast.
+
 Numeric attention values: parity unpinned by the paper (it prints no attention
 value); every function here is pinned by the library routine, closed forms and
 invariants named above, in tests/test_oracle_pins.py.
@@ -56,7 +62,23 @@ def rope(x: np.ndarray, pos, theta: float) -> np.ndarray:
     return np.concatenate([lo * c - hi * s, hi * c + lo * s], axis=-1)
 
 
-def standalone_attend(k_raw: np.ndarray, v_raw: np.ndarray, q_raw: np.ndarray, theta: float) -> np.ndarray:
+def quantize_e4m3(x: np.ndarray) -> np.ndarray:
+    """Nearest e4m3 number (ties to even mantissa, magnitudes beyond 448 saturate to 448), returned as fp64.
+
+    e4m3: value = (-1)^s * 2^(e-7) * (1 + m/8) for exponent field e in 1..15 and mantissa m in 0..7 (e = 15, m = 7 is
+    not a number and never produced), and (-1)^s * 2^-6 * m/8 for e = 0.  So the numbers are spaced 2^(E-3) apart in
+    the binade [2^E, 2^(E+1)), E >= -6, and 2^-9 apart below 2^-6.
+    """
+    x = np.asarray(x, dtype=np.float64)
+    a = np.abs(x)
+    E = np.floor(np.log2(np.maximum(a, 2.0 ** -6)))  # binade of |x|; everything below 2^-6 uses the subnormal spacing
+    step = 2.0 ** (E - 3)
+    q = np.rint(a / step) * step  # np.rint rounds halves to even
+    return np.sign(x) * np.minimum(q, 448.0)
+
+
+def standalone_attend(k_raw: np.ndarray, v_raw: np.ndarray, q_raw: np.ndarray, theta: float,
+                      kv_e4m3: bool = False) -> np.ndarray:
     """Attention output of the LAST token of one standalone prompt.
 
     k_raw, v_raw: [T, D] raw keys / values of the prompt's T tokens (context tokens,
@@ -64,12 +86,15 @@ def standalone_attend(k_raw: np.ndarray, v_raw: np.ndarray, q_raw: np.ndarray, t
     token whose query is evaluated).  q_raw: [H, D] raw queries of that last token
     for the H query heads that share this KV head.  Ordinary positions 0..T-1; the
     query sits at T-1 and sees all T keys (itself included).  Returns [H, D] fp64.
+    kv_e4m3: the rotated keys and the values are the e4m3 numbers nearest to them (the 8-bit cache variant).
     """
     k_raw = np.asarray(k_raw, dtype=np.float64)
     v = np.asarray(v_raw, dtype=np.float64)
     q_raw = np.asarray(q_raw, dtype=np.float64)
     T, D = k_raw.shape
     k = rope(k_raw, np.arange(T), theta)
+    if kv_e4m3:
+        k, v = quantize_e4m3(k), quantize_e4m3(v)
     q = rope(q_raw, np.full(q_raw.shape[0], T - 1), theta)
     z = (q @ k.T) / np.sqrt(D)
     z = z - z.max(axis=-1, keepdims=True)
@@ -285,12 +310,12 @@ def tuple_inputs(wl, b: int, k: int, s: int, layer: int, kv_head: int, ctx_cache
 
 
 def attend_tuple(wl, b: int, k: int, s: int, layer: int, kv_head: int, ctx_cache: dict | None = None,
-                 step_cache: dict | None = None) -> np.ndarray:
+                 step_cache: dict | None = None, kv_e4m3: bool = False) -> np.ndarray:
     """Oracle output for question k (global id) of prompt b at decode step s, one layer, all query heads of one KV
     head: [G, D] fp64 -- `standalone_attend` on the standalone prompt assembled by `tuple_inputs`.  Pinned by the
     dense-mask formulation assembled independently in the tests (the equivalence of Sec. 4.2)."""
     k_raw, v_raw, q_raw = tuple_inputs(wl, b, k, s, layer, kv_head, ctx_cache, step_cache)
-    return standalone_attend(k_raw, v_raw, q_raw, wl.geom.rope_theta)
+    return standalone_attend(k_raw, v_raw, q_raw, wl.geom.rope_theta, kv_e4m3)
 
 
 def prefill_tuple(wl, b: int, k: int | None, layer: int, kv_head: int) -> np.ndarray:

@@ -446,3 +446,74 @@ def test_prefill_tuple_equals_header_rows_of_the_dense_formulation(shared_len):
                 rows_x = [i for i, t in enumerate(tag) if t[0] == "x" and t[1] == b and t[2] == k - int(wl.q_begin[b])]
                 np.testing.assert_allclose(orc.prefill_tuple(wl, b, k, 0, kv_head), dense[rows_x][:, hs], atol=1e-12,
                                            rtol=0)
+
+
+# --------------------------------------------------------------------------- the 8-bit cache variant
+def _all_e4m3_values():
+    """Every finite e4m3 number from the bit fields (1-4-3, bias 7, subnormals, S.1111.111 is not a number)."""
+    vals = []
+    for code in range(256):
+        sgn = -1.0 if code & 0x80 else 1.0
+        e, m = (code >> 3) & 0xF, code & 0x7
+        if e == 15 and m == 7:
+            continue
+        vals.append(sgn * (2.0 ** -6 * m / 8 if e == 0 else 2.0 ** (e - 7) * (1 + m / 8)))
+    return np.array(sorted(set(vals)))
+
+
+def test_quantize_e4m3_hand_values():
+    # spacing 1/32 in [1/4, 1/2): 0.3 -> 10/32; 2^-5 in [1/8, 1/4); ties go to the even mantissa; 448 is the largest
+    x = np.array([0.3, 0.2, 1.0625, 1.1875, 17.0, 19.0, 300.0, 447.0, 464.0, 1e6, -0.3, 0.0, 2.0 ** -10, 3 * 2.0 ** -10,
+                  0.0009])
+    want = np.array([0.3125, 0.203125, 1.0, 1.25, 16.0, 20.0, 288.0, 448.0, 448.0, 448.0, -0.3125, 0.0, 0.0,
+                     2.0 ** -8, 0.0])
+    np.testing.assert_array_equal(orc.quantize_e4m3(x), want)
+
+
+def test_quantize_e4m3_is_the_nearest_code_by_enumeration():
+    codes = _all_e4m3_values()
+    assert codes.size == 253 and codes.max() == 448.0 and codes[codes > 0].min() == 2.0 ** -9  # +-126 and one zero
+    np.testing.assert_array_equal(orc.quantize_e4m3(codes), codes)  # fixed points
+    rng = np.random.default_rng(5)
+    x = np.concatenate([rng.normal(size=4000), rng.normal(size=2000) * 40, rng.normal(size=2000) * 0.01,
+                        rng.uniform(-460, 460, size=2000)])
+    q = orc.quantize_e4m3(x)
+    d = np.abs(x[:, None] - codes[None, :])
+    best = d.min(axis=1)
+    assert np.all(np.isin(q, codes))
+    np.testing.assert_allclose(np.abs(x - q), best, rtol=0, atol=1e-15)  # no code is nearer
+    # exact midpoints between neighbouring codes go to the code with the even mantissa (the even multiple of the
+    # smaller code's spacing)
+    mid = (codes[:-1] + codes[1:]) / 2
+    qm = orc.quantize_e4m3(mid)
+    lo, hi = codes[:-1], codes[1:]
+    step = np.minimum(np.abs(hi - lo), 2.0 ** 5)
+    k_lo = np.rint(np.abs(lo) / step)
+    even_is_lo = (k_lo % 2 == 0)
+    # around zero and across binades the rule is the same in units of the finer spacing
+    np.testing.assert_array_equal(qm, np.where(even_is_lo, lo, hi))
+
+
+def test_quantize_e4m3_equals_the_library_cast():
+    rng = np.random.default_rng(6)
+    x = np.concatenate([rng.normal(size=20000), rng.normal(size=5000) * 30, rng.normal(size=5000) * 0.02])
+    x = x[np.abs(x) < 440].astype(np.float32)  # the library's cast does not saturate the same way beyond the range
+    lib = torch.from_numpy(x).to(torch.float8_e4m3fn).to(torch.float64).numpy()
+    np.testing.assert_array_equal(orc.quantize_e4m3(x.astype(np.float64)), lib)
+
+
+def test_attend_e4m3_is_plain_attention_over_the_quantised_cache():
+    rng = np.random.default_rng(8)
+    T, D, H, theta = 37, 64, 4, 1e4
+    k_raw, v_raw, q_raw = rng.normal(size=(T, D)), rng.normal(size=(T, D)), rng.normal(size=(H, D))
+    got = orc.standalone_attend(k_raw, v_raw, q_raw, theta, kv_e4m3=True)
+    # independent route: the library's float8 cast of the rotated keys and of the values, then torch SDPA's last row
+    k8 = torch.from_numpy(orc.rope(k_raw, np.arange(T), theta).astype(np.float32)).to(torch.float8_e4m3fn).double()
+    v8 = torch.from_numpy(v_raw.astype(np.float32)).to(torch.float8_e4m3fn).double()
+    q = torch.from_numpy(orc.rope(q_raw, np.full(H, T - 1), theta))
+    want = torch.nn.functional.scaled_dot_product_attention(q[None], k8[None], v8[None])[0].numpy()
+    np.testing.assert_allclose(got, want, rtol=1e-10, atol=1e-12)
+    # and it differs from the unquantised result by what 3 mantissa bits cost, not by more
+    exact = orc.standalone_attend(k_raw, v_raw, q_raw, theta)
+    err = np.abs(got - exact).max() / np.sqrt((exact ** 2).mean())
+    assert 1e-3 < err < 0.5
