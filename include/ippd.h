@@ -64,6 +64,17 @@ extern "C" {
                                       (a wait on a phase not yet complete fails at once: IPPD_ERR_TIMEOUT) */
 #define IPPD_OPT_PROFILE 5         /* N > 0: bracket the attention, merge and STEP-append kernels of every N-th step
                                       (counted from this call: steps 0, N, 2N, ...) with CUDA events; 0: off */
+#define IPPD_OPT_KV_DTYPE 6        /* element type of the cache: IPPD_KV_BF16 (default) or IPPD_KV_E4M3.  Only before
+                                      ippd_bind_cache (ippd_cache_bytes follows it); tensor-core path only.
+                                      IPPD_KV_E4M3, a bandwidth variant that is not part of the paper: the rotated
+                                      key and the value are stored as e4m3 numbers (1-4-3 bits, bias 7, largest
+                                      magnitude 448, round to nearest even, saturating; no scale factor), half the
+                                      bytes per token.  Scores and outputs are those of exact attention over the
+                                      stored numbers, to the same tolerance as the bf16 cache: inside the kernel the
+                                      query rows and the probabilities enter the 8-bit tensor-core products as sums
+                                      of two e4m3 terms.  All entry points work unchanged on such a cache. */
+#define IPPD_KV_BF16 0
+#define IPPD_KV_E4M3 1
 
 typedef struct {
   int32_t n_layers;

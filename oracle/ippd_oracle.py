@@ -103,7 +103,8 @@ def standalone_attend(k_raw: np.ndarray, v_raw: np.ndarray, q_raw: np.ndarray, t
     return p @ v
 
 
-def standalone_prefill(k_raw: np.ndarray, v_raw: np.ndarray, q_raw: np.ndarray, theta: float) -> np.ndarray:
+def standalone_prefill(k_raw: np.ndarray, v_raw: np.ndarray, q_raw: np.ndarray, theta: float,
+                       kv_e4m3: bool = False) -> np.ndarray:
     """Causal self-attention of ONE standalone prompt, every row (the prefill of a triplet prompted alone).
 
     k_raw, v_raw: [T, D] raw keys / values of the prompt's T tokens; q_raw: [T, H, D] raw queries of the same tokens
@@ -117,6 +118,8 @@ def standalone_prefill(k_raw: np.ndarray, v_raw: np.ndarray, q_raw: np.ndarray, 
     T, D = k_raw.shape
     pos = np.arange(T)
     k = rope(k_raw, pos, theta)
+    if kv_e4m3:  # the 8-bit cache variant: every row reads the stored numbers, its own token's included
+        k, v = quantize_e4m3(k), quantize_e4m3(v)
     out = np.empty_like(q_raw)
     causal = np.tril(np.ones((T, T), dtype=bool))
     for h in range(q_raw.shape[1]):
@@ -318,7 +321,7 @@ def attend_tuple(wl, b: int, k: int, s: int, layer: int, kv_head: int, ctx_cache
     return standalone_attend(k_raw, v_raw, q_raw, wl.geom.rope_theta, kv_e4m3)
 
 
-def prefill_tuple(wl, b: int, k: int | None, layer: int, kv_head: int) -> np.ndarray:
+def prefill_tuple(wl, b: int, k: int | None, layer: int, kv_head: int, kv_e4m3: bool = False) -> np.ndarray:
     """Oracle prefill outputs of the header rows of one standalone prompt, one layer, all query heads of one KV head.
 
     k = a global question id: the prompt is (instruction p, context c_b, question x_k); returns the rows of the
@@ -339,5 +342,5 @@ def prefill_tuple(wl, b: int, k: int | None, layer: int, kv_head: int) -> np.nda
         kq, vq = wl.question_kv(k, layer)
         ks.append(kq[:, kv_head]); vs.append(vq[:, kv_head]); qs.append(wl.question_q(k, layer)[:, hs])
     cat = lambda ts: np.concatenate([t.double().numpy() for t in ts])
-    out = standalone_prefill(cat(ks), cat(vs), cat(qs), g.rope_theta)
+    out = standalone_prefill(cat(ks), cat(vs), cat(qs), g.rope_theta, kv_e4m3)
     return out if k is None else out[-int(wl.q_len[k]):]

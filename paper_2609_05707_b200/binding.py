@@ -22,7 +22,8 @@ BF16, F32 = 0, 1
 TILE_TOKENS = 128
 STATIC_SCRATCH_BYTES = 64 << 20
 APPEND_CONTEXT, APPEND_QUESTION, APPEND_STEP, APPEND_SHARED, APPEND_HEADER = 0, 1, 2, 3, 4
-OPT_KERNEL, OPT_LAYERS_PER_CALL, OPT_TILES_PER_SPLIT, OPT_WAIT_LIMIT_US, OPT_PROFILE = 1, 2, 3, 4, 5
+OPT_KERNEL, OPT_LAYERS_PER_CALL, OPT_TILES_PER_SPLIT, OPT_WAIT_LIMIT_US, OPT_PROFILE, OPT_KV_DTYPE = 1, 2, 3, 4, 5, 6
+KV_BF16, KV_E4M3 = 0, 1
 
 EXPORTS = ["ippd_build_layout", "ippd_build_layout_shared", "ippd_layout_tables", "ippd_cache_bytes", "ippd_bind_cache", "ippd_set_option",
            "ippd_begin_step", "ippd_step_descriptor_bytes", "ippd_append_kv", "ippd_workspace_bytes", "ippd_decode_attention", "ippd_decode_step", "ippd_decode_step_grouped", "ippd_prefill_attention", "ippd_decode_attention_static",

@@ -175,6 +175,7 @@ static IppdDev make_dev(const ippd_layout* L) {
   d.D = L->h.geom.head_dim;
   d.max_pos = L->h.max_pos;
   d.shared_len = L->h.shared_len;
+  d.kv8 = L->h.opt_kv_dtype == IPPD_KV_E4M3;
   return d;
 }
 
@@ -231,6 +232,7 @@ extern "C" int ippd_set_option(ippd_layout_t* L, int32_t key, int64_t value) {
   switch (key) {
     case IPPD_OPT_KERNEL:
       if (value < 0 || value > 2) { ippd_set_error("ippd_set_option: kernel path not available"); return IPPD_ERR_INVALID_ARG; }
+      if (value == 1 && L->h.opt_kv_dtype == IPPD_KV_E4M3) { ippd_set_error("ippd_set_option: the 8-bit cache needs the tensor-core path"); return IPPD_ERR_INVALID_ARG; }
       L->h.opt_kernel = (int32_t)value;
       break;
     case IPPD_OPT_LAYERS_PER_CALL:
@@ -247,6 +249,12 @@ extern "C" int ippd_set_option(ippd_layout_t* L, int32_t key, int64_t value) {
       L->profile_steps = 0;
       L->profile = false;
       return IPPD_OK;
+    case IPPD_OPT_KV_DTYPE:
+      if (value != IPPD_KV_BF16 && value != IPPD_KV_E4M3) { ippd_set_error("ippd_set_option: unknown cache element type"); return IPPD_ERR_INVALID_ARG; }
+      if (L->bound) { ippd_set_error("ippd_set_option: the cache element type is fixed once a cache is bound"); return IPPD_ERR_INVALID_ARG; }
+      if (value == IPPD_KV_E4M3 && L->h.kernel_path() < 2) { ippd_set_error("ippd_set_option: the 8-bit cache needs the tensor-core path"); return IPPD_ERR_INVALID_ARG; }
+      L->h.opt_kv_dtype = (int32_t)value;
+      break;
     case IPPD_OPT_WAIT_LIMIT_US:
       if (value < 0 || value > 60000000) { ippd_set_error("ippd_set_option: bad wait limit"); return IPPD_ERR_INVALID_ARG; }
       L->h.opt_wait_limit_us = value;
@@ -545,12 +553,13 @@ extern "C" int ippd_append_kv(ippd_layout_t* L, int32_t layer_begin, int32_t lay
   }
   const bool prof = kind == IPPD_APPEND_STEP;
   if (prof) prof_mark(L, 2, true, stream);
+  const bool kv8 = h.opt_kv_dtype == IPPD_KV_E4M3;
   if (D == 128)
-    CUDA_TRY(launch_pdl(ippd_append_kernel<128>, grid, dim3(256), 0, stream, d, L->step_dev, a, layer_begin,
-                        (const __nv_bfloat16*)k_raw, (const __nv_bfloat16*)v_raw));
+    CUDA_TRY(launch_pdl(kv8 ? ippd_append_kernel<128, true> : ippd_append_kernel<128, false>, grid, dim3(256), 0, stream,
+                        d, L->step_dev, a, layer_begin, (const __nv_bfloat16*)k_raw, (const __nv_bfloat16*)v_raw));
   else
-    CUDA_TRY(launch_pdl(ippd_append_kernel<64>, grid, dim3(256), 0, stream, d, L->step_dev, a, layer_begin,
-                        (const __nv_bfloat16*)k_raw, (const __nv_bfloat16*)v_raw));
+    CUDA_TRY(launch_pdl(kv8 ? ippd_append_kernel<64, true> : ippd_append_kernel<64, false>, grid, dim3(256), 0, stream,
+                        d, L->step_dev, a, layer_begin, (const __nv_bfloat16*)k_raw, (const __nv_bfloat16*)v_raw));
   if (prof) prof_mark(L, 2, false, stream);
   CUDA_TRY(cudaGetLastError());
   L->launches++;
@@ -648,8 +657,10 @@ static int launch_attention(ippd_layout* L, const IppdDev& d, int layer_begin, i
     if (!attr_set[dev]) {
       CUDA_TRY(cudaFuncSetAttribute(ippd_attn_mma_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                     MmaCfg<D>::SMEM));
-      CUDA_TRY(cudaFuncSetAttribute(ippd_attn_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                    tc_smem_bytes<D>()));
+      CUDA_TRY(cudaFuncSetAttribute(ippd_attn_tc_kernel<D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    tc_smem_bytes<D, false>()));
+      CUDA_TRY(cudaFuncSetAttribute(ippd_attn_tc_kernel<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    tc_smem_bytes<D, true>()));
       attr_set[dev] = true;
     }
   }
@@ -674,8 +685,10 @@ static int launch_attention(ippd_layout* L, const IppdDev& d, int layer_begin, i
     a.k_step = (const __nv_bfloat16*)k_step;
     a.v_step = (const __nv_bfloat16*)v_step;
     if (marks) prof_mark(L, 0, true, stream);
-    CUDA_TRY(launch_pdl(ippd_attn_tc_kernel<D>, dim3(grid), dim3(IPPD_TC_THREADS), (size_t)tc_smem_bytes<D>(), stream, d,
-                        S, a, (const __nv_bfloat16*)q_raw, out, part_o, part_ml));
+    const bool kv8 = L->h.opt_kv_dtype == IPPD_KV_E4M3;
+    CUDA_TRY(launch_pdl(kv8 ? ippd_attn_tc_kernel<D, true> : ippd_attn_tc_kernel<D, false>, dim3(grid),
+                        dim3(IPPD_TC_THREADS), (size_t)(kv8 ? tc_smem_bytes<D, true>() : tc_smem_bytes<D, false>()),
+                        stream, d, S, a, (const __nv_bfloat16*)q_raw, out, part_o, part_ml));
     if (marks) prof_mark(L, 0, false, stream);
     CUDA_TRY(cudaGetLastError());
     L->launches++;
@@ -978,14 +991,13 @@ extern "C" int ippd_read_probe(ippd_layout_t* L, int32_t layer_begin, int32_t la
   a.layer_count = layer_count;
   IppdDev d = make_dev(L);
   const int D = h.geom.head_dim;
-  const size_t smem = (size_t)IPPD_TC_NBUF * IPPD_TILE_TOKENS * D * 2 + IPPD_TC_NBUF * sizeof(uint64_t);
-  if (D == 128) {
-    CUDA_TRY(cudaFuncSetAttribute(ippd_read_probe_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    ippd_read_probe_kernel<128><<<grid, 64, smem, stream>>>(d, L->step_dev, a);
-  } else {
-    CUDA_TRY(cudaFuncSetAttribute(ippd_read_probe_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    ippd_read_probe_kernel<64><<<grid, 64, smem, stream>>>(d, L->step_dev, a);
-  }
+  const bool kv8 = h.opt_kv_dtype == IPPD_KV_E4M3;
+  auto kern = D == 128 ? (kv8 ? ippd_read_probe_kernel<128, true> : ippd_read_probe_kernel<128, false>)
+                       : (kv8 ? ippd_read_probe_kernel<64, true> : ippd_read_probe_kernel<64, false>);
+  const size_t nbuf = kv8 ? TcCfg<128, true>::NBUF : TcCfg<128, false>::NBUF;
+  const size_t smem = nbuf * h.tile_bytes() + nbuf * sizeof(uint64_t);
+  CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  kern<<<grid, 64, smem, stream>>>(d, L->step_dev, a);
   CUDA_TRY(cudaGetLastError());
   L->launches++;
   return IPPD_OK;

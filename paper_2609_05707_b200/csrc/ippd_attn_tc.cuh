@@ -41,6 +41,18 @@
 #define IPPD_TC_MAX_CTAS 192   // upper bound of the persistent grid (one CTA per SM)
 #define IPPD_TC_RESCALE_THRESHOLD 8.0f  // log2 units: the reference maximum may lag by up to 2^8
 
+// Sizes that depend on the cache's element type.  KV8: keys and values are e4m3 bytes (half the bytes per token, so
+// almost twice as many buffers of half the size); the products then run on the 8-bit tensor-core kind, with the query
+// rows and the probabilities each split into two e4m3 terms (value = hi + lo) so that they keep bf16-like precision.
+template <int D, bool KV8>
+struct TcCfg {
+  static constexpr int GB = (KV8 ? D / 16 : D / 8) * 128;  // bytes of an 8-token group (one row of core matrices)
+  static constexpr int TILE_BYTES = 16 * GB;               // 128 tokens
+  static constexpr int NBUF = KV8 ? 13 : IPPD_TC_NBUF;
+  static constexpr int NMETA = KV8 ? 8 : 5;
+  static constexpr int PV_TOKENS = KV8 ? 32 : 16;          // tokens one P V product consumes
+};
+
 struct IppdTcArgs {
   const int32_t* rb_tile_begin;  // [n_rb+1] first tile of each row block inside one (layer, head) sequence
   const IppdTcTile* tiles;       // [T1] tiles of one (layer, head) sequence
@@ -89,6 +101,20 @@ __device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint
       "r"(a_tmem), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(acc)
       : "memory");
 }
+// The 8-bit kind: fp32 accumulate, e4m3 x e4m3 (format code 0), A K-major in TMEM (four values per 32-bit column),
+// B K- or MN-major in shared memory.
+__device__ __forceinline__ uint32_t tc_idesc8(int M, int N, int b_mn_major) {
+  return (1u << 4) | ((uint32_t)b_mn_major << 16) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+__device__ __forceinline__ void tc_mma_ts8(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t b_hi,
+                                           uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t.reg .b64 db;\n\t"
+      "mov.b64 db, {%2, %3};\n\tsetp.ne.b32 p, %5, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], [%1], db, %4, p;\n\t}" ::"r"(d_tmem),
+      "r"(a_tmem), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(acc)
+      : "memory");
+}
 __device__ __forceinline__ void tc_commit(uint64_t* bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
                : "memory");
@@ -134,6 +160,8 @@ __device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sy
         "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])     \
       : "r"(taddr)                                                                                               \
       : "memory")
+#define TC_ST2(taddr, r) \
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x2.b32 [%2], {%0,%1};" ::"r"(r[0]), "r"(r[1]), "r"(taddr) : "memory")
 #define TC_ST4(taddr, r)                                                                                       \
   asm volatile("tcgen05.st.sync.aligned.32x32b.x4.b32 [%4], {%0,%1,%2,%3};" ::"r"(r[0]), "r"(r[1]), "r"(r[2]), \
                "r"(r[3]), "r"(taddr)                                                                            \
@@ -174,7 +202,7 @@ __device__ __forceinline__ bool tc_next_segment(const IppdTcArgs& a, const IppdS
   return true;
 }
 
-#define IPPD_TC_NMETA 5
+#define IPPD_TC_NMETA 5  // (bf16 cache; the 8-bit variant has its own count in TcCfg)
 // Per-tile description staged in shared memory by the producer warp.  The producer starts tile t + 5 only after the
 // P V product of tile t has released its V buffer (7 ring buffers, two per tile), and every reader of tile t's entry
 // is done by then, so five entries suffice.  For a packed branch tile, [c0[a], c1[a]) are the columns question `a` of
@@ -185,8 +213,10 @@ struct TcMeta {
   uint8_t c0[64], c1[64];
 };
 
-struct TcShared {
-  uint64_t kv_full[IPPD_TC_NBUF], kv_empty[IPPD_TC_NBUF];
+template <int NBUF, int NMETA>
+struct TcSharedT {
+  static constexpr int kNMeta = NMETA;
+  uint64_t kv_full[NBUF], kv_empty[NBUF];
   uint64_t s_full[2], p_full[2];
   uint64_t pv_done[2];
   uint64_t o_free, q_full;
@@ -195,12 +225,14 @@ struct TcShared {
   volatile int abort_flag;
   uint32_t app_done;     // the append warp has finished the packed tiles with index (in the CTA's slice) below this
   unsigned short xmax[2][4][IPPD_TC_ROWS];  // [tile parity][warpgroup][row]: bf16 bits of the quarter-row maxima
-  TcMeta meta[IPPD_TC_NMETA];
+  TcMeta meta[NMETA];
 };
+using TcShared = TcSharedT<IPPD_TC_NBUF, IPPD_TC_NMETA>;
 
-template <int D>
+template <int D, bool KV8 = false>
 constexpr int tc_smem_bytes() {
-  return IPPD_TC_NBUF * 16 * (D / 8) * 128 + (int)sizeof(TcShared);
+  using C = TcCfg<D, KV8>;
+  return C::NBUF * C::TILE_BYTES + (int)sizeof(TcSharedT<C::NBUF, C::NMETA>);
 }
 
 
@@ -256,11 +288,12 @@ __device__ __forceinline__ bool tc_wait_appended(const uint32_t* counter, uint32
 // full.  Lane 0 owns the barriers and the context copies, lane i < n_pieces fetches piece i of a packed tile; the
 // tile's description is left in shared memory for the other roles (published by the K buffer's mbarrier, which this
 // warp arrives on afterwards).  SH needs kv_full[], kv_empty[], meta[], app_done and abort_flag.
-template <int D, int NBUF, class SH>
+template <int D, int NBUF, class SH, bool KV8 = false>
 __device__ __forceinline__ void tc_producer_role(const IppdDev& L, const IppdStepDev& S, const IppdTcArgs& A, SH* sh,
                                                  uint8_t* ring, long long g0, long long g1, int lane) {
-  constexpr int GB = (D / 8) * 128;
+  constexpr int GB = TcCfg<D, KV8>::GB;
   constexpr int TILE_BYTES = 16 * GB;
+  constexpr int PVG = TcCfg<D, KV8>::PV_TOKENS / 8;  // 8-token groups one P V product consumes
   const int Hkv = L.Hkv;
   long long g = g0;
   TcSegment sg;
@@ -284,7 +317,7 @@ __device__ __forceinline__ void tc_producer_role(const IppdDev& L, const IppdSte
         ti_next = A.tiles[t + 1];
         if (lane < ti_next.n_pieces) pc_next = A.pieces[ti_next.piece_begin + lane];
       }
-      TcMeta& mt = sh->meta[tc % IPPD_TC_NMETA];
+      TcMeta& mt = sh->meta[tc % SH::kNMeta];
       if (lane == 0) { mt.rows = ti.rows; mt.n_pieces = ti.n_pieces; }
       if (ti.n_pieces > 0) {
         // column window of every question in this tile: its pieces sit on adjacent lanes, the first gives c0 and
@@ -322,11 +355,13 @@ __device__ __forceinline__ void tc_producer_role(const IppdDev& L, const IppdSte
         ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
         if (!ok) break;
         uint8_t* dst = ring + buf * TILE_BYTES;
-        if (kv == 1 && (groups & 1)) {
-          // The P V product works in steps of 16 rows: the 8 rows after an odd number of fetched groups are not
-          // written by the copies below and would be stale shared memory; P is zero there, but 0 * NaN = NaN.
+        if (kv == 1 && (groups % PVG) != 0) {
+          // The P V product works in steps of 16 (8-bit cache: 32) rows: the rows between the fetched groups and the
+          // end of the last step are not written by the copies below and would be stale shared memory; P is zero
+          // there, but 0 * NaN = NaN.
           uint4* z = reinterpret_cast<uint4*>(dst + groups * GB);
-          for (int idx = lane; idx < GB / 16; idx += 32) z[idx] = make_uint4(0, 0, 0, 0);
+          const int n16 = (PVG - groups % PVG) * (GB / 16);
+          for (int idx = lane; idx < n16; idx += 32) z[idx] = make_uint4(0, 0, 0, 0);
           asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
           __syncwarp();
         }
@@ -334,11 +369,11 @@ __device__ __forceinline__ void tc_producer_role(const IppdDev& L, const IppdSte
         __syncwarp();
         if (ti.n_pieces <= 0) {
           if (lane == 0)
-            bulk_g2s(dst, L.cache + ippd_tile_addr(L, layer, sg.head, ti.pool_tile, kv), (uint32_t)groups * GB,
+            bulk_g2s(dst, L.cache + ippd_tile_addr<KV8>(L, layer, sg.head, ti.pool_tile, kv), (uint32_t)groups * GB,
                      &sh->kv_full[buf]);
         } else if (lane < ti.n_pieces) {
           bulk_g2s(dst + (pc.row0 >> 3) * GB,
-                   L.cache + ippd_tile_addr(L, layer, sg.head, pc.src_tile, kv) + (size_t)pc.src_group * GB,
+                   L.cache + ippd_tile_addr<KV8>(L, layer, sg.head, pc.src_tile, kv) + (size_t)pc.src_group * GB,
                    (uint32_t)pc.n_groups * GB, &sh->kv_full[buf]);
         }
       }
@@ -358,7 +393,7 @@ __device__ __forceinline__ void tc_producer_role(const IppdDev& L, const IppdSte
 // Append role (one warp, only when the call carries the step's raw K/V): walks the CTA's slice ahead of the producer
 // and, for every packed branch piece that holds the token fed at this step, rotates its key (RoPE) and writes K~ and V
 // into the piece's cache slot; the producer fetches a packed tile only after its slots are in place.
-template <int D, class SH>
+template <int D, class SH, bool KV8 = false>
 __device__ __forceinline__ void tc_append_role(const IppdDev& L, const IppdStepDev& S, const IppdTcArgs& A, SH* sh,
                                                long long g0, long long g1, int lane) {
   const int Hkv = L.Hkv;
@@ -395,8 +430,9 @@ __device__ __forceinline__ void tc_append_role(const IppdDev& L, const IppdStepD
           if (have) {
             const int a = rb.act_begin + a_local;
             const size_t row = (((size_t)sg.ll * S.A + a) * Hkv + sg.head) * D + c * 8;
-            ippd_rope_store_pair<D>(L, A.k_step + row, A.v_step + row, S.act_pos[a], c,
-                                    ippd_tile_addr(L, layer, sg.head, src_tile, 0), src_group * 8 + new_tok - 1);
+            ippd_rope_store_pair<D, KV8>(L, A.k_step + row, A.v_step + row, S.act_pos[a], c,
+                                         ippd_tile_addr<KV8>(L, layer, sg.head, src_tile, 0),
+                                         src_group * 8 + new_tok - 1);
           }
           for (int i = 0; i < TPP && todo; ++i) todo &= todo - 1;
         }
@@ -414,16 +450,18 @@ __device__ __forceinline__ void tc_append_role(const IppdDev& L, const IppdStepD
 
 #include "ippd_attn_tc_softmax.cuh"
 
-template <int D>
+template <int D, bool KV8 = false>
 __global__ void __launch_bounds__(IPPD_TC_THREADS, 1)
 ippd_attn_tc_kernel(IppdDev L, IppdStepDev S, IppdTcArgs A, const __nv_bfloat16* __restrict__ q_raw,
                     void* __restrict__ out, float* __restrict__ part_o, float* __restrict__ part_ml) {
-  constexpr int DC = D / 8;                 // 16-byte chunks per row
-  constexpr int GB = DC * 128;              // bytes of an 8-row group
-  constexpr int TILE_BYTES = 16 * GB;       // 128 rows
+  using Cfg = TcCfg<D, KV8>;
+  using SH = TcSharedT<Cfg::NBUF, Cfg::NMETA>;
+  constexpr int NBUF = Cfg::NBUF;
+  constexpr int GB = Cfg::GB;                  // bytes of an 8-row group
+  constexpr int TILE_BYTES = Cfg::TILE_BYTES;  // 128 rows
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   uint8_t* ring = smem_raw;  // NBUF buffers of 128 rows
-  TcShared* sh = reinterpret_cast<TcShared*>(ring + IPPD_TC_NBUF * TILE_BYTES);
+  SH* sh = reinterpret_cast<SH*>(ring + NBUF * TILE_BYTES);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int Hkv = L.Hkv;
@@ -431,7 +469,7 @@ ippd_attn_tc_kernel(IppdDev L, IppdStepDev S, IppdTcArgs A, const __nv_bfloat16*
   const long long g0 = A.cut[blockIdx.x], g1 = A.cut[blockIdx.x + 1];
 
   if (tid == 0) {
-    for (int i = 0; i < IPPD_TC_NBUF; ++i) { mbar_init(&sh->kv_full[i], 1); mbar_init(&sh->kv_empty[i], 1); }
+    for (int i = 0; i < NBUF; ++i) { mbar_init(&sh->kv_full[i], 1); mbar_init(&sh->kv_empty[i], 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(&sh->s_full[i], 1); mbar_init(&sh->p_full[i], 16); }
     for (int i = 0; i < 2; ++i) mbar_init(&sh->pv_done[i], 1);
     mbar_init(&sh->drain[0], 1);
@@ -458,14 +496,14 @@ ippd_attn_tc_kernel(IppdDev L, IppdStepDev S, IppdTcArgs A, const __nv_bfloat16*
   const uint32_t tS0 = tmem, tO = tmem + 256, tQ = tmem + 384;
 
   if (warp == 0) {
-    tc_producer_role<D, IPPD_TC_NBUF>(L, S, A, sh, ring, g0, g1, lane);
+    tc_producer_role<D, NBUF, SH, KV8>(L, S, A, sh, ring, g0, g1, lane);
   } else if (warp == 1) {
     // =========================== P V issuer (one lane) ===========================
     // O += P(j) V(j): P from TMEM (the head of S buffer j & 1), V from ring slot 2j+1 (MN-major).
     if (lane == 0) {
       const uint32_t ring_lo_v = tc_desc_lo(smem_u32(ring), GB);  // d chunks 128 B apart, 8-token groups GB apart
       const uint32_t hi_v = tc_desc_hi(128);
-      const uint32_t idesc_pv = tc_idesc(128, D, 1);
+      const uint32_t idesc_pv = KV8 ? tc_idesc8(128, D, 1) : tc_idesc(128, D, 1);
       long long g = g0;
       TcSegment sg;
       uint32_t jt = 0;  // tiles processed so far by this CTA
@@ -474,7 +512,7 @@ ippd_attn_tc_kernel(IppdDev L, IppdStepDev S, IppdTcArgs A, const __nv_bfloat16*
       while (ok && tc_next_segment(A, S, Hkv, g0, g1, g, sg)) {
         const int nt = sg.t_end - sg.t_begin;
         for (int i = 0; i < nt; ++i, ++jt) {
-          const uint32_t nb = 2 * jt + 1, buf = nb % IPPD_TC_NBUF, ph = (nb / IPPD_TC_NBUF) & 1;
+          const uint32_t nb = 2 * jt + 1, buf = nb % NBUF, ph = (nb / NBUF) & 1;
           if (!tc_wait(&sh->kv_full[buf], ph, L, sh)) { ok = false; break; }
           if (!tc_wait(&sh->p_full[jt & 1], (jt >> 1) & 1, L, sh)) { ok = false; break; }
           if (i == 0 && nseg > 0) {
@@ -484,9 +522,19 @@ ippd_attn_tc_kernel(IppdDev L, IppdStepDev S, IppdTcArgs A, const __nv_bfloat16*
           tc_fence_after();
           const uint32_t v_lo = ring_lo_v + buf * (TILE_BYTES >> 4);
           const uint32_t a_tmem = tS0 + (jt & 1) * 128;
-          const int ksteps = (sh->meta[jt % IPPD_TC_NMETA].rows + 15) >> 4;
-          for (int k = 0; k < ksteps; ++k)
-            tc_mma_ts(tO, a_tmem + k * 8, v_lo + k * (2 * GB >> 4), hi_v, idesc_pv, (i > 0 || k > 0) ? 1u : 0u);
+          if constexpr (KV8) {
+            // P = P_hi + P_lo, two e4m3 rows (columns +0 and +32 of the S buffer, four tokens per column), each
+            // against the same V tile, 32 tokens per product
+            const int ksteps = (sh->meta[jt % SH::kNMeta].rows + 31) >> 5;
+            for (int half = 0; half < 2; ++half)
+              for (int k = 0; k < ksteps; ++k)
+                tc_mma_ts8(tO, a_tmem + half * 32 + k * 8, v_lo + k * (4 * GB >> 4), hi_v, idesc_pv,
+                           (i > 0 || half > 0 || k > 0) ? 1u : 0u);
+          } else {
+            const int ksteps = (sh->meta[jt % SH::kNMeta].rows + 15) >> 4;
+            for (int k = 0; k < ksteps; ++k)
+              tc_mma_ts(tO, a_tmem + k * 8, v_lo + k * (2 * GB >> 4), hi_v, idesc_pv, (i > 0 || k > 0) ? 1u : 0u);
+          }
           tc_commit(&sh->kv_empty[buf]);
           tc_commit(&sh->pv_done[jt & 1]);
         }
@@ -497,7 +545,7 @@ ippd_attn_tc_kernel(IppdDev L, IppdStepDev S, IppdTcArgs A, const __nv_bfloat16*
       mbar_wait_ns(&sh->drain[0], 0, L, IPPD_DRAIN_LIMIT_NS);
     }
   } else if (warp == IPPD_TC_WARP_APPEND) {
-    tc_append_role<D>(L, S, A, sh, g0, g1, lane);
+    tc_append_role<D, SH, KV8>(L, S, A, sh, g0, g1, lane);
   } else if (warp == IPPD_TC_WARP_S_ISSUER) {
     // =========================== S issuer (one lane) ===========================
     // S(j) = Q~ K(j)^T: Q~ from TMEM, K from ring slot 2j (K-major), into S buffer j & 1.  That buffer held P(j-2),
@@ -524,16 +572,27 @@ ippd_attn_tc_kernel(IppdDev L, IppdStepDev S, IppdTcArgs A, const __nv_bfloat16*
         if (!tc_wait(&sh->q_full, nseg & 1, L, sh)) break;
         const uint32_t a_tmem = tQ + (nseg & 1) * 64;
         for (int i = 0; i < nt; ++i, ++jt) {
-          const uint32_t nb = 2 * jt, buf = nb % IPPD_TC_NBUF, ph = (nb / IPPD_TC_NBUF) & 1;
+          const uint32_t nb = 2 * jt, buf = nb % NBUF, ph = (nb / NBUF) & 1;
           if (!tc_wait(&sh->kv_full[buf], ph, L, sh)) { ok = false; break; }
           if (jt >= 2 && !tc_wait(&sh->pv_done[jt & 1], ((jt - 2) >> 1) & 1, L, sh)) { ok = false; break; }
           tc_fence_after();
-          const int rows_i = sh->meta[jt % IPPD_TC_NMETA].rows;  // published by the K buffer's barrier
-          const uint32_t idesc = tc_idesc(128, (rows_i + 15) & ~15, 0);
+          const int rows_i = sh->meta[jt % SH::kNMeta].rows;  // published by the K buffer's barrier
           const uint32_t k_lo = ring_lo + buf * (TILE_BYTES >> 4);
           const uint32_t d_tmem = tS0 + (jt & 1) * 128;
+          if constexpr (KV8) {
+            // Q~ = Q~_hi + Q~_lo, two e4m3 rows (columns +0 and +D/4 of the Q~ buffer), each against the same K tile,
+            // 32 values of d per product
+            const uint32_t idesc = tc_idesc8(128, (rows_i + 15) & ~15, 0);
 #pragma unroll
-          for (int k = 0; k < D / 16; ++k) tc_mma_ts(d_tmem, a_tmem + k * 8, k_lo + k * 16, hi_k, idesc, k > 0);
+            for (int half = 0; half < 2; ++half)
+#pragma unroll
+              for (int k = 0; k < D / 32; ++k)
+                tc_mma_ts8(d_tmem, a_tmem + half * (D / 4) + k * 8, k_lo + k * 16, hi_k, idesc, (half > 0 || k > 0));
+          } else {
+            const uint32_t idesc = tc_idesc(128, (rows_i + 15) & ~15, 0);
+#pragma unroll
+            for (int k = 0; k < D / 16; ++k) tc_mma_ts(d_tmem, a_tmem + k * 8, k_lo + k * 16, hi_k, idesc, k > 0);
+          }
           tc_commit(&sh->kv_empty[buf]);
           tc_commit(&sh->s_full[jt & 1]);
         }
@@ -544,7 +603,7 @@ ippd_attn_tc_kernel(IppdDev L, IppdStepDev S, IppdTcArgs A, const __nv_bfloat16*
     }
   } else {
     // =========================== softmax / correction / epilogue (warps 2..17) ===========================
-    tc_softmax_role<D>(L, S, A, sh, tmem, g0, g1, q_raw, out, part_o, part_ml);
+    tc_softmax_role<D, SH, KV8>(L, S, A, sh, tmem, g0, g1, q_raw, out, part_o, part_ml);
   }
 
   // ---- teardown: every role gets here (all waits are bounded) ----

@@ -33,6 +33,47 @@ __device__ __forceinline__ void tc_exp8(const uint32_t* s, float scale, float m,
           (__uint_as_float(p[3] << 16) + __uint_as_float(p[3] & 0xFFFF0000u));
 }
 
+// The 8-bit cache variant: the probabilities enter the P V product as two e4m3 rows, P = P_hi + P_lo (P_hi the
+// nearest e4m3 number, P_lo the nearest to the rest), which keeps about 8 significant bits; the exponent is biased so
+// that the row's largest probability lies in [2^(BIAS), 2^(BIAS + THRESHOLD)] = [16, 256] and the smallest one that
+// survives (2^-9, the e4m3 subnormal step) is 2^-13 of it or less.  The bias multiplies numerator and row sum alike.
+#define IPPD_TC8_BIAS 4.0f
+#define IPPD_TC8_RESCALE_THRESHOLD 4.0f
+// exp2(s*scale - m) for 8 consecutive S values -> 2 words of P_hi and 2 of P_lo (four e4m3 values each, the first in
+// the lowest byte); the row sum is taken over the unrounded values.
+__device__ __forceinline__ void tc_exp8_f8(const uint32_t* s, float scale, float m, uint32_t* p_hi, uint32_t* p_lo,
+                                           float& acc0, float& acc1) {
+  uint32_t h16[4], l16[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const float e0 = fast_exp2(fmaf(__uint_as_float(s[2 * i]), scale, -m));
+    const float e1 = fast_exp2(fmaf(__uint_as_float(s[2 * i + 1]), scale, -m));
+    if (i & 1) acc1 += e0 + e1; else acc0 += e0 + e1;
+    const __half2 e = __floats2half2_rn(e0, e1);
+    const __nv_fp8x2_storage_t hi = __nv_cvt_halfraw2_to_fp8x2(static_cast<__half2_raw>(e), __NV_SATFINITE, __NV_E4M3);
+    const __half2 back = __half2(__nv_cvt_fp8x2_to_halfraw2(hi, __NV_E4M3));
+    const __half2 rest = __hsub2(e, back);  // exact: the two are within a factor of two of each other
+    const __nv_fp8x2_storage_t lo = __nv_cvt_halfraw2_to_fp8x2(static_cast<__half2_raw>(rest), __NV_SATFINITE, __NV_E4M3);
+    h16[i] = hi;
+    l16[i] = lo;
+  }
+  p_hi[0] = h16[0] | (h16[1] << 16);
+  p_hi[1] = h16[2] | (h16[3] << 16);
+  p_lo[0] = l16[0] | (l16[1] << 16);
+  p_lo[1] = l16[2] | (l16[3] << 16);
+}
+// Four floats -> the e4m3 numbers nearest to them (a word) and nearest to what is left (another word).
+__device__ __forceinline__ void tc_split_e4m3x4(float a, float b, float c, float d, uint32_t& hi, uint32_t& lo) {
+  const __nv_fp8x2_storage_t h0 = __nv_cvt_float2_to_fp8x2(make_float2(a, b), __NV_SATFINITE, __NV_E4M3);
+  const __nv_fp8x2_storage_t h1 = __nv_cvt_float2_to_fp8x2(make_float2(c, d), __NV_SATFINITE, __NV_E4M3);
+  const float2 b0 = __half22float2(__half2(__nv_cvt_fp8x2_to_halfraw2(h0, __NV_E4M3)));
+  const float2 b1 = __half22float2(__half2(__nv_cvt_fp8x2_to_halfraw2(h1, __NV_E4M3)));
+  const __nv_fp8x2_storage_t l0 = __nv_cvt_float2_to_fp8x2(make_float2(a - b0.x, b - b0.y), __NV_SATFINITE, __NV_E4M3);
+  const __nv_fp8x2_storage_t l1 = __nv_cvt_float2_to_fp8x2(make_float2(c - b1.x, d - b1.y), __NV_SATFINITE, __NV_E4M3);
+  hi = (uint32_t)h0 | ((uint32_t)h1 << 16);
+  lo = (uint32_t)l0 | ((uint32_t)l1 << 16);
+}
+
 // Upper 16 bits of the smallest bf16 value >= x: the exchanged maximum must not be smaller than the true one, so that
 // every probability stays <= 1.  (Positive: round the magnitude up; negative: truncate it.)
 __device__ __forceinline__ unsigned short tc_bf16_ceil_bits(float x) {
@@ -65,9 +106,9 @@ __device__ __noinline__ void tc_quad_give_up(const int32_t* rb_tile_begin, int n
   for (long long k = 0; k < owed; ++k) tc_quad_sync(warp);
 }
 
-template <int D>
+template <int D, class SH = TcShared, bool KV8 = false>
 __device__ __forceinline__ void tc_softmax_role(const IppdDev& L, const IppdStepDev& S, const IppdTcArgs& A,
-                                                TcShared* sh, uint32_t tmem, long long g0, long long g1,
+                                                SH* sh, uint32_t tmem, long long g0, long long g1,
                                                 const __nv_bfloat16* __restrict__ q_raw, void* __restrict__ out,
                                                 float* __restrict__ part_o, float* __restrict__ part_ml) {
   constexpr int DQ = D / IPPD_TC_NWG;  // output columns per warpgroup (32 or 16)
@@ -85,7 +126,87 @@ __device__ __forceinline__ void tc_softmax_role(const IppdDev& L, const IppdStep
   // Stages this warpgroup's part of Q~ of segment `sq` into TMEM buffer `qbuf` (the A operand of S = Q~ K^T: lane = row,
   // column c holds the bf16 pair (2c, 2c+1) of the row) and signals the MMA warp.  The buffer was last read by the S
   // MMAs of the segment before the previous one, which are long complete.
+  // 8-bit cache variant: the row is scaled by a power of two that brings its largest magnitude to [64, 182) (from the
+  // largest raw magnitude: the rotation grows a value by less than sqrt 2), split into Q~_hi + Q~_lo (two e4m3 rows,
+  // four values per column; hi at columns [0, D/4), lo at [D/4, D/2)), and the inverse factor goes into the score
+  // scale of the row, which the call returns.
+  auto stage_q8 = [&](const TcSegment& sq, uint32_t qbuf) -> float {
+    constexpr int NV = D / 8;  // values per warpgroup and rotation half (16 or 8)
+    const IppdRowBlock rb = S.rbs[sq.rb];
+    const int nrows = rb.n_act * G;
+    uint32_t hl[NV / 4], hh[NV / 4], ll_[NV / 4], lh[NV / 4];
+    float inv_f = 1.f;
+    if (row < nrows) {
+      const int j = row - my_q * G, ai = rb.act_begin + my_q;
+      const int pos = S.act_pos[ai];
+      const __nv_bfloat16* qp = q_raw + (((size_t)sq.ll * S.A + ai) * L.Hq + sq.head * G + j) * D;
+      uint32_t mx = 0;  // largest magnitude of the raw row, as bf16 bits (they order like integers)
+#pragma unroll
+      for (int c = 0; c < D / 8; ++c) {
+        const uint4 w = *reinterpret_cast<const uint4*>(qp + c * 8);
+        const uint32_t ws[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) mx = max(mx, max(ws[e] & 0x7FFFu, (ws[e] >> 16) & 0x7FFFu));
+      }
+      int field = 260 - (int)(mx >> 7);  // exponent field of 2^(6 - floor(log2 max))
+      field = min(250, max(4, field));
+      const float f = __uint_as_float((uint32_t)field << 23);
+      inv_f = __uint_as_float((uint32_t)(254 - field) << 23);
+      const float2* cs = L.rope + (size_t)pos * (D / 2);
+      float ql[NV], qh[NV];
+#pragma unroll
+      for (int cc = 0; cc < NV / 8; ++cc) {
+        const int c = wg * (NV / 8) + cc;  // 16-byte chunk c of the raw row and its rotation partner c + D/16
+        uint4 lo = *reinterpret_cast<const uint4*>(qp + c * 8);
+        uint4 hi = *reinterpret_cast<const uint4*>(qp + c * 8 + D / 2);
+        const __nv_bfloat162* pl = reinterpret_cast<const __nv_bfloat162*>(&lo);
+        const __nv_bfloat162* ph = reinterpret_cast<const __nv_bfloat162*>(&hi);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          float2 c0 = cs[c * 8 + 2 * e], c1 = cs[c * 8 + 2 * e + 1];
+          float l0 = __bfloat162float(pl[e].x) * f, l1 = __bfloat162float(pl[e].y) * f;
+          float h0 = __bfloat162float(ph[e].x) * f, h1 = __bfloat162float(ph[e].y) * f;
+          ql[cc * 8 + 2 * e] = l0 * c0.x - h0 * c0.y;
+          ql[cc * 8 + 2 * e + 1] = l1 * c1.x - h1 * c1.y;
+          qh[cc * 8 + 2 * e] = h0 * c0.x + l0 * c0.y;
+          qh[cc * 8 + 2 * e + 1] = h1 * c1.x + l1 * c1.y;
+        }
+      }
+#pragma unroll
+      for (int e = 0; e < NV / 4; ++e) {
+        tc_split_e4m3x4(ql[4 * e], ql[4 * e + 1], ql[4 * e + 2], ql[4 * e + 3], hl[e], ll_[e]);
+        tc_split_e4m3x4(qh[4 * e], qh[4 * e + 1], qh[4 * e + 2], qh[4 * e + 3], hh[e], lh[e]);
+      }
+    } else {
+#pragma unroll
+      for (int e = 0; e < NV / 4; ++e) { hl[e] = 0u; hh[e] = 0u; ll_[e] = 0u; lh[e] = 0u; }
+    }
+    // values d = (NV wg ..) sit in columns NV/4 * wg .., their rotation partners D/8 columns further; lo rows D/4 further
+    const uint32_t tq = tQ + qbuf * 64 + lane_base + wg * (NV / 4);
+    if constexpr (NV == 16) {
+      { uint32_t* w = hl; TC_ST4(tq, w); }
+      { uint32_t* w = hh; TC_ST4(tq + D / 8, w); }
+      { uint32_t* w = ll_; TC_ST4(tq + D / 4, w); }
+      { uint32_t* w = lh; TC_ST4(tq + D / 4 + D / 8, w); }
+    } else {
+      { uint32_t* w = hl; TC_ST2(tq, w); }
+      { uint32_t* w = hh; TC_ST2(tq + D / 8, w); }
+      { uint32_t* w = ll_; TC_ST2(tq + D / 4, w); }
+      { uint32_t* w = lh; TC_ST2(tq + D / 4 + D / 8, w); }
+    }
+    tc_wait_st();
+    tc_fence_before();
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&sh->q_full);
+    return scale_log2 * inv_f;
+  };
+  float sc_cur = scale_log2, sc_next = scale_log2;  // score scale of my row (8-bit variant: with the row's factor)
+  (void)sc_next;
   auto stage_q = [&](const TcSegment& sq, uint32_t qbuf) {
+    if constexpr (KV8) {
+      sc_next = stage_q8(sq, qbuf);
+      return;
+    }
     const IppdRowBlock rb = S.rbs[sq.rb];
     const int nrows = rb.n_act * G;
     uint32_t wlo[NW], whi[NW];  // rotated pairs d in [2*NW*wg, 2*NW*(wg+1)) and the same + D/2
@@ -139,6 +260,8 @@ __device__ __forceinline__ void tc_softmax_role(const IppdDev& L, const IppdStep
   }
   if (have) stage_q(sg, 0);
   while (have) {
+    if constexpr (KV8) sc_cur = sc_next;  // staged with this segment's Q~ (before the loop or during the last segment)
+    const float sc = KV8 ? sc_cur : scale_log2;
     const IppdRowBlock rb = S.rbs[sg.rb];
     const int nrows = rb.n_act * G;
     // A context tile is seen whole by every query row, so a warp with at least one query row takes the path without
@@ -153,7 +276,7 @@ __device__ __forceinline__ void tc_softmax_role(const IppdDev& L, const IppdStep
       if (!tc_wait(&sh->s_full[jt & 1], (jt >> 1) & 1, L, sh)) { tc_quad_give_up(A.rb_tile_begin, S.n_rb, A.T1, g0 + gofs, g1, nt - i + 3, warp); return; }
       tc_fence_after();
       // the tile's description was staged by the producer before its K copy, which S(jt) has consumed
-      const TcMeta& meta = sh->meta[jt % IPPD_TC_NMETA];
+      const TcMeta& meta = sh->meta[jt % SH::kNMeta];
       const int tile_rows = meta.rows, n_pieces = meta.n_pieces;
       const int base = wg * IPPD_TC_CW;              // my first column
       const bool part_used = tile_rows > base;       // the P V product reads my columns of the P row
@@ -221,7 +344,7 @@ __device__ __forceinline__ void tc_softmax_role(const IppdDev& L, const IppdStep
             }
           }
         }
-        mloc = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3)) * scale_log2;
+        mloc = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3)) * sc;
       }
       // exchange the quarter-row maxima, rounded up to bf16 so that all four owners derive the same reference; the
       // barrier also orders every owner's S loads before the P stores below, which overwrite S columns of other owners
@@ -236,7 +359,8 @@ __device__ __forceinline__ void tc_softmax_role(const IppdDev& L, const IppdStep
                    fmaxf(__uint_as_float((uint32_t)b2 << 16), __uint_as_float((uint32_t)b3 << 16)));
       }
       // lazy rescale: keep the old reference unless the row's maximum grew past the threshold (or it is the first)
-      const bool grow = mt > m_ref + IPPD_TC_RESCALE_THRESHOLD || (m_ref == -INFINITY && mt > -INFINITY);
+      const bool grow = mt > m_ref + (KV8 ? IPPD_TC8_RESCALE_THRESHOLD : IPPD_TC_RESCALE_THRESHOLD) ||
+                        (m_ref == -INFINITY && mt > -INFINITY);
       float alpha = 1.f;
       if (grow) {
         alpha = fast_exp2(m_ref - mt);  // 0 when this is the row's first visible tile
@@ -257,6 +381,25 @@ __device__ __forceinline__ void tc_softmax_role(const IppdDev& L, const IppdStep
       // ---- my 16 packed words of the P row (zeros where my row sees nothing) ----
       if (part_used) {
         uint32_t p[IPPD_TC_CW / 2];
+        if constexpr (KV8) {
+          // p[0..7]: my 32 tokens of P_hi (columns 8 wg .. of the S buffer), p[8..15]: of P_lo (32 columns further)
+          if (warp_any) {
+            const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref - IPPD_TC8_BIAS;
+            float a0 = 0.f, a1 = 0.f;
+#pragma unroll
+            for (int e = 0; e < IPPD_TC_CW; e += 8) {
+              if (e >= wlo && e < whi) tc_exp8_f8(s + e, sc, m_use, p + e / 4, p + 8 + e / 4, a0, a1);
+              else { p[e / 4] = 0u; p[e / 4 + 1] = 0u; p[8 + e / 4] = 0u; p[8 + e / 4 + 1] = 0u; }
+            }
+            l_sum += a0 + a1;
+          } else {
+#pragma unroll
+            for (int e = 0; e < IPPD_TC_CW / 2; ++e) p[e] = 0u;
+          }
+          const uint32_t tP8 = tS0 + (jt & 1) * 128 + wg * (IPPD_TC_CW / 4) + lane_base;
+          { uint32_t* w = p; TC_ST8(tP8, w); }
+          { uint32_t* w = p + 8; TC_ST8(tP8 + 32, w); }
+        } else {
         if (warp_any) {
           const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;  // rows that see nothing yet: exp2(-inf) = 0
           float a0 = 0.f, a1 = 0.f;
@@ -271,6 +414,7 @@ __device__ __forceinline__ void tc_softmax_role(const IppdDev& L, const IppdStep
           for (int e = 0; e < IPPD_TC_CW / 2; ++e) p[e] = 0u;
         }
         TC_ST16(tP, p);
+        }
       }
       tc_wait_st();  // the P words and a possible O rescale
       tc_fence_before();

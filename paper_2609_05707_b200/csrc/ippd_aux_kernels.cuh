@@ -18,7 +18,9 @@ __global__ void ippd_rope_table_kernel(float2* table, int max_pos, int D, double
 // and the same two chunks of V.  k_src / v_src point at chunk c of the token's raw row; `k_tile` is the byte offset of
 // the K half of the destination cache tile (its V half follows it), `u` the token's row inside the tile.  Cache tile
 // layout (K and V alike): [token/8][d/8][token%8][d%8] bf16, i.e. 8x8 blocks of 128 contiguous bytes.
-template <int D>
+// KV8: the rotated key and the value are stored as e4m3 bytes, [token/8][d/16][token%8][d%16] (8x16 blocks of 128
+// bytes); a thread's 8 values are half of a block row.
+template <int D, bool KV8 = false>
 __device__ __forceinline__ void ippd_rope_store_pair(const IppdDev& L, const __nv_bfloat16* __restrict__ k_src,
                                                      const __nv_bfloat16* __restrict__ v_src, int pos, int c,
                                                      size_t k_tile, int u) {
@@ -44,24 +46,56 @@ __device__ __forceinline__ void ippd_rope_store_pair(const IppdDev& L, const __n
   const float2* cs = L.rope + (size_t)pos * (D / 2) + c * 8;
   const __nv_bfloat162* pl = reinterpret_cast<const __nv_bfloat162*>(&klo);
   const __nv_bfloat162* ph = reinterpret_cast<const __nv_bfloat162*>(&khi);
-  uint4 olo, ohi;
-  uint32_t* wl = reinterpret_cast<uint32_t*>(&olo);
-  uint32_t* wh = reinterpret_cast<uint32_t*>(&ohi);
+  if constexpr (KV8) {
+    constexpr int GB8 = (D / 16) * 128;
+    float kl[8], kh[8];
 #pragma unroll
-  for (int e = 0; e < 4; ++e) {
-    float2 c0 = cs[2 * e], c1 = cs[2 * e + 1];
-    float l0 = __bfloat162float(pl[e].x), l1 = __bfloat162float(pl[e].y);
-    float h0 = __bfloat162float(ph[e].x), h1 = __bfloat162float(ph[e].y);
-    wl[e] = pack_bf16(l0 * c0.x - h0 * c0.y, l1 * c1.x - h1 * c1.y);
-    wh[e] = pack_bf16(h0 * c0.x + l0 * c0.y, h1 * c1.x + l1 * c1.y);
+    for (int e = 0; e < 4; ++e) {
+      float2 c0 = cs[2 * e], c1 = cs[2 * e + 1];
+      float l0 = __bfloat162float(pl[e].x), l1 = __bfloat162float(pl[e].y);
+      float h0 = __bfloat162float(ph[e].x), h1 = __bfloat162float(ph[e].y);
+      kl[2 * e] = l0 * c0.x - h0 * c0.y;
+      kl[2 * e + 1] = l1 * c1.x - h1 * c1.y;
+      kh[2 * e] = h0 * c0.x + l0 * c0.y;
+      kh[2 * e + 1] = h1 * c1.x + l1 * c1.y;
+    }
+    const __nv_bfloat16* vl = reinterpret_cast<const __nv_bfloat16*>(&vlo);
+    const __nv_bfloat16* vh = reinterpret_cast<const __nv_bfloat16*>(&vhi);
+    auto f = [](__nv_bfloat16 x) { return __bfloat162float(x); };
+    const uint2 k_lo8 = make_uint2(pack_e4m3x4(kl[0], kl[1], kl[2], kl[3]), pack_e4m3x4(kl[4], kl[5], kl[6], kl[7]));
+    const uint2 k_hi8 = make_uint2(pack_e4m3x4(kh[0], kh[1], kh[2], kh[3]), pack_e4m3x4(kh[4], kh[5], kh[6], kh[7]));
+    const uint2 v_lo8 = make_uint2(pack_e4m3x4(f(vl[0]), f(vl[1]), f(vl[2]), f(vl[3])),
+                                   pack_e4m3x4(f(vl[4]), f(vl[5]), f(vl[6]), f(vl[7])));
+    const uint2 v_hi8 = make_uint2(pack_e4m3x4(f(vh[0]), f(vh[1]), f(vh[2]), f(vh[3])),
+                                   pack_e4m3x4(f(vh[4]), f(vh[5]), f(vh[6]), f(vh[7])));
+    // values d = 8c.. sit in 16-value block c/2, half c%2; the rotation partners D/2 further in block D/32 + c/2
+    const size_t in_tile = (size_t)(u >> 3) * GB8 + (size_t)(u & 7) * 16 + (size_t)(c & 1) * 8;
+    char* kdst = L.cache + k_tile + in_tile;
+    char* vdst = kdst + (size_t)IPPD_TILE_TOKENS * D;  // the V half of the tile follows its K half
+    *reinterpret_cast<uint2*>(kdst + (c >> 1) * 128) = k_lo8;
+    *reinterpret_cast<uint2*>(kdst + (D / 32 + (c >> 1)) * 128) = k_hi8;
+    *reinterpret_cast<uint2*>(vdst + (c >> 1) * 128) = v_lo8;
+    *reinterpret_cast<uint2*>(vdst + (D / 32 + (c >> 1)) * 128) = v_hi8;
+  } else {
+    uint4 olo, ohi;
+    uint32_t* wl = reinterpret_cast<uint32_t*>(&olo);
+    uint32_t* wh = reinterpret_cast<uint32_t*>(&ohi);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      float2 c0 = cs[2 * e], c1 = cs[2 * e + 1];
+      float l0 = __bfloat162float(pl[e].x), l1 = __bfloat162float(pl[e].y);
+      float h0 = __bfloat162float(ph[e].x), h1 = __bfloat162float(ph[e].y);
+      wl[e] = pack_bf16(l0 * c0.x - h0 * c0.y, l1 * c1.x - h1 * c1.y);
+      wh[e] = pack_bf16(h0 * c0.x + l0 * c0.y, h1 * c1.x + l1 * c1.y);
+    }
+    const size_t in_tile = (size_t)(u >> 3) * GB + (size_t)(u & 7) * 16;
+    char* kdst = L.cache + k_tile + in_tile;
+    char* vdst = kdst + (size_t)IPPD_TILE_TOKENS * D * 2;  // the V half of the tile follows its K half
+    *reinterpret_cast<uint4*>(kdst + c * 128) = olo;
+    *reinterpret_cast<uint4*>(kdst + (c + CP) * 128) = ohi;
+    *reinterpret_cast<uint4*>(vdst + c * 128) = vlo;
+    *reinterpret_cast<uint4*>(vdst + (c + CP) * 128) = vhi;
   }
-  const size_t in_tile = (size_t)(u >> 3) * GB + (size_t)(u & 7) * 16;
-  char* kdst = L.cache + k_tile + in_tile;
-  char* vdst = kdst + (size_t)IPPD_TILE_TOKENS * D * 2;  // the V half of the tile follows its K half
-  *reinterpret_cast<uint4*>(kdst + c * 128) = olo;
-  *reinterpret_cast<uint4*>(kdst + (c + CP) * 128) = ohi;
-  *reinterpret_cast<uint4*>(vdst + c * 128) = vlo;
-  *reinterpret_cast<uint4*>(vdst + (c + CP) * 128) = vhi;
 }
 
 #define IPPD_APPEND_INLINE 64
@@ -85,7 +119,7 @@ struct IppdAppendArgs {
 };
 
 // One thread moves one (token, KV head, pair of 16-byte chunks c and c + D/16), see ippd_rope_store_pair.
-template <int D>
+template <int D, bool KV8 = false>
 __global__ void __launch_bounds__(256)
 ippd_append_kernel(IppdDev L, IppdStepDev S, IppdAppendArgs a, int layer_begin,
                    const __nv_bfloat16* __restrict__ k_raw, const __nv_bfloat16* __restrict__ v_raw) {
@@ -164,7 +198,7 @@ ippd_append_kernel(IppdDev L, IppdStepDev S, IppdAppendArgs a, int layer_begin,
     return;
   }
   size_t src = (((size_t)ll * a.n_tokens + tok) * L.Hkv + head) * D + c * 8;
-  ippd_rope_store_pair<D>(L, k_raw + src, v_raw + src, pos, c, ippd_tile_addr(L, layer, head, tile, 0), u);
+  ippd_rope_store_pair<D, KV8>(L, k_raw + src, v_raw + src, pos, c, ippd_tile_addr<KV8>(L, layer, head, tile, 0), u);
 }
 
 // Token descriptor of the mask export: kind 0 = context token, 1 = question token, 2 = answer token.

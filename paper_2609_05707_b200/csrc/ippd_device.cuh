@@ -1,6 +1,7 @@
 // Device-side primitives (inline PTX for sm_100a) and parameter structs of the IPPD kernels.
 #pragma once
 #include <cuda_bf16.h>
+#include <cuda_fp8.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -26,6 +27,7 @@ struct IppdDev {
   long long wait_limit_ns;
   int n_layers, Hq, Hkv, G, D, max_pos;
   int shared_len;  // tokens of the instruction shared by all prompts (positions 0 .. shared_len-1, tiles from 0)
+  int kv8;         // 1: the cache holds e4m3 bytes (IPPD_OPT_KV_DTYPE)
 };
 
 // Per-step arrays (device pointers into the step blob).
@@ -38,8 +40,10 @@ struct IppdStepDev {
   int A, n_rb, n_units, RB;
 };
 
+// Byte offset of the K (kv = 0) or V (kv = 1) half of a cache tile.  KV8: the cache holds e4m3 bytes, not bf16.
+template <bool KV8 = false>
 __device__ __forceinline__ size_t ippd_tile_addr(const IppdDev& L, int layer, int head, long long tile, int kv) {
-  size_t tile_bytes = (size_t)IPPD_TILE_TOKENS * L.D * 2;
+  size_t tile_bytes = (size_t)IPPD_TILE_TOKENS * L.D * (KV8 ? 1 : 2);
   return ((((size_t)layer * L.Hkv + head) * (size_t)L.n_tiles + (size_t)tile) * 2 + kv) * tile_bytes;
 }
 
@@ -158,6 +162,12 @@ __device__ __forceinline__ float fast_exp2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
+}
+// Four floats -> four e4m3 bytes (round to nearest even, saturating at 448), a in the lowest byte.
+__device__ __forceinline__ uint32_t pack_e4m3x4(float a, float b, float c, float d) {
+  const uint32_t lo = __nv_cvt_float2_to_fp8x2(make_float2(a, b), __NV_SATFINITE, __NV_E4M3);
+  const uint32_t hi = __nv_cvt_float2_to_fp8x2(make_float2(c, d), __NV_SATFINITE, __NV_E4M3);
+  return lo | (hi << 16);
 }
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);

@@ -92,9 +92,11 @@ struct IppdHostLayout {
   int32_t max_pos = 0;
   // options
   int32_t opt_kernel = 0, opt_layers_per_call = 0, opt_tiles_per_split = 0;
+  int32_t opt_kv_dtype = IPPD_KV_BF16;
   int64_t opt_wait_limit_us = 2000000;
 
-  size_t tile_bytes() const { return (size_t)IPPD_TILE_TOKENS * geom.head_dim * 2; }
+  // K (or V) half of a 128-token cache tile
+  size_t tile_bytes() const { return (size_t)IPPD_TILE_TOKENS * geom.head_dim * (opt_kv_dtype == IPPD_KV_E4M3 ? 1 : 2); }
   size_t cache_bytes() const {
     return (size_t)geom.n_layers * geom.n_kv_heads * (size_t)n_tiles * 2 * tile_bytes();
   }

@@ -19,7 +19,7 @@ from .workloads import Workload
 class Runner:
     def __init__(self, wl: Workload, device: str = "cuda:0", out_dtype: int = B.BF16, kernel: int = 0,
                  layers_per_call: Optional[int] = None, tiles_per_split: int = 0, branch_align: int = B.TILE_TOKENS,
-                 fused: bool = True):
+                 fused: bool = True, kv_dtype: int = B.KV_BF16):
         if not torch.cuda.is_available():
             raise RuntimeError("the IPPD library needs a CUDA device; there is no CPU fallback")
         self.wl = wl
@@ -32,6 +32,9 @@ class Runner:
         self.layout = B.Layout(self.geom, wl.ctx_len, wl.q_count, wl.q_len, wl.max_new, shared_len=wl.shared_len)
         if kernel:
             self.layout.set_option(B.OPT_KERNEL, kernel)
+        self.kv_dtype = kv_dtype
+        if kv_dtype != B.KV_BF16:
+            self.layout.set_option(B.OPT_KV_DTYPE, kv_dtype)  # before the cache is sized and bound
         if layers_per_call:
             self.layout.set_option(B.OPT_LAYERS_PER_CALL, layers_per_call)
         if tiles_per_split:

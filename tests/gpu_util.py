@@ -62,7 +62,10 @@ class PoisonedRunner(Runner):
     def __init__(self, *a, **kw):
         self._guarded = []
         super().__init__(*a, **kw)
-        self.cache.view(torch.int16).fill_(0x7F7F)
+        if self.kv_dtype == B.KV_E4M3:
+            self.cache.fill_(0x7E)  # 448, the largest finite e4m3 number (0x7F is not a number)
+        else:
+            self.cache.view(torch.int16).fill_(0x7F7F)
         self.workspace.fill_(0xFF)
         torch.cuda.synchronize()
 
@@ -89,10 +92,10 @@ class PoisonedRunner(Runner):
         self.guards_intact()
 
 
-def oracle_step(wl, s, layer, kv_head, cache=None, step_cache=None, qids=None):
+def oracle_step(wl, s, layer, kv_head, cache=None, step_cache=None, qids=None, kv_e4m3=False):
     """Oracle outputs of the active questions (or the given subset) at step s: {qid: [G, D]}."""
     qids = wl.active(s) if qids is None else qids
-    return {int(k): orc.attend_tuple(wl, int(wl.prompt_of[k]), int(k), s, layer, kv_head, cache, step_cache)
+    return {int(k): orc.attend_tuple(wl, int(wl.prompt_of[k]), int(k), s, layer, kv_head, cache, step_cache, kv_e4m3)
             for k in qids}
 
 
@@ -105,7 +108,7 @@ def compare_step(runner, s, layers, kv_heads, cache, what, rel=True, absolute=Tr
     got, want = [], []
     for layer in layers:
         for h in kv_heads:
-            ref = oracle_step(wl, s, layer, h, cache)
+            ref = oracle_step(wl, s, layer, h, cache, kv_e4m3=runner.kv_dtype == B.KV_E4M3)
             for i, k in enumerate(act):
                 got.append(out[layer, i, h * G:(h + 1) * G])
                 want.append(ref[int(k)])

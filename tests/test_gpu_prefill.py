@@ -23,7 +23,7 @@ def _header_index(wl):
     return ctx0, q0, t
 
 
-def _compare_header(wl, out, layers, heads, ctx_rows=None, questions=None, what="prefill"):
+def _compare_header(wl, out, layers, heads, ctx_rows=None, questions=None, what="prefill", kv_e4m3=False):
     """out: [n_layers, n_hdr, Hq, D] numpy.  ctx_rows: {b: positions inside (instruction + context)} or None = all;
     questions: ids or None = all."""
     G, P = wl.geom.group, wl.shared_len
@@ -40,7 +40,7 @@ def _compare_header(wl, out, layers, heads, ctx_rows=None, questions=None, what=
                 Lb = int(wl.ctx_len[b])
                 if P + Lb == 0:
                     continue  # no instruction and an empty context: the prompt has question rows only
-                ref = orc.prefill_tuple(wl, b, None, layer, h)  # rows of p and c_b
+                ref = orc.prefill_tuple(wl, b, None, layer, h, kv_e4m3)  # rows of p and c_b
                 pick = range(P + Lb) if rows is None else rows
                 for r in pick:
                     if r < P:
@@ -49,7 +49,7 @@ def _compare_header(wl, out, layers, heads, ctx_rows=None, questions=None, what=
                     else:
                         got.append(out[layer, ctx0[b] + r - P, hs]); want.append(ref[r])
             for k in (range(wl.n_questions) if questions is None else questions):
-                ref = orc.prefill_tuple(wl, int(wl.prompt_of[k]), int(k), layer, h)
+                ref = orc.prefill_tuple(wl, int(wl.prompt_of[k]), int(k), layer, h, kv_e4m3)
                 for j in range(int(wl.q_len[k])):
                     got.append(out[layer, q0[k] + j, hs]); want.append(ref[j])
     # rows that see only a handful of keys have outputs of size ~1: the absolute gate is stated for averages over

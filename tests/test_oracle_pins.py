@@ -517,3 +517,13 @@ def test_attend_e4m3_is_plain_attention_over_the_quantised_cache():
     exact = orc.standalone_attend(k_raw, v_raw, q_raw, theta)
     err = np.abs(got - exact).max() / np.sqrt((exact ** 2).mean())
     assert 1e-3 < err < 0.5
+
+
+def test_prefill_e4m3_last_row_is_the_e4m3_decode_row():
+    rng = np.random.default_rng(9)
+    T, D, H, theta = 21, 64, 2, 1e4
+    k_raw, v_raw, q_raw = rng.normal(size=(T, D)), rng.normal(size=(T, D)), rng.normal(size=(T, H, D))
+    full = orc.standalone_prefill(k_raw, v_raw, q_raw, theta, kv_e4m3=True)
+    for t in (0, 5, T - 1):  # row t of the prefill is the decode row of the prompt cut after token t
+        row = orc.standalone_attend(k_raw[:t + 1], v_raw[:t + 1], q_raw[t], theta, kv_e4m3=True)
+        np.testing.assert_allclose(full[t], row, rtol=1e-10, atol=1e-12)
