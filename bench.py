@@ -206,13 +206,19 @@ class ConfigBench:
 
     def __init__(self, name, dev, kernel, max_resident_bytes=24e9, n_layers=0):
         import torch
+        from paper_2609_05707_b200 import binding as B
         from paper_2609_05707_b200 import workloads as W
         from paper_2609_05707_b200.runner import Runner
         self.torch = torch
-        self.wl = wl = W.make_workload(name, n_layers or None)
+        base, _, kv = name.partition("/")  # "C3/e4m3": workload C3 on the 8-bit cache variant
+        if kv not in ("", "e4m3"):
+            raise SystemExit(f"unknown cache variant in {name!r}")
+        self.kv_elem_bytes = 1 if kv == "e4m3" else 2
+        self.wl = wl = W.make_workload(base, n_layers or None)
         self.g = g = wl.geom
         self.dev = dev
-        self.run = Runner(wl, dev, kernel=kernel, layers_per_call=g.n_layers)
+        self.run = Runner(wl, dev, kernel=kernel, layers_per_call=g.n_layers,
+                          kv_dtype=B.KV_E4M3 if kv == "e4m3" else B.KV_BF16)
         self.run.load_header()
         self.run.append_all_steps()
         self.run.check()
@@ -342,7 +348,7 @@ class ConfigBench:
             lay.read_probe(0, g.n_layers, self.run.stream)
             e1.record()
             torch.cuda.synchronize()
-            b = self.wl.step_bytes(s)
+            b = self.wl.step_bytes(s, self.kv_elem_bytes)
             tot_ms += e0.elapsed_time(e1)
             tot_bytes += b["context"] + b["branch"]
         self.run.check()
@@ -366,13 +372,14 @@ def measure_config(name, args, dev, peaks, sync, want_layer_modes, rank_world):
     prof_steps = [timed[i % len(timed)] for i in range(max(16, len(timed)))]
     prof = cb.profile(prof_steps)
     n_att = max(1, prof["n_attention"])
-    bytes_total = sum(wl.step_bytes(s)["total"] for s in prof_steps)
+    kvb = cb.kv_elem_bytes
+    bytes_total = sum(wl.step_bytes(s, kvb)["total"] for s in prof_steps)
     flops_total = sum(wl.step_flops(s) for s in prof_steps)
     call_ms = prof["attention_ms"] + prof["merge_ms"]  # the ippd_decode_attention / ippd_decode_step time
     achieved = bytes_total / (call_ms * 1e-3) / 1e9 if call_ms > 0 else 0.0
     kernel_gbs = bytes_total / (prof["attention_ms"] * 1e-3) / 1e9 if prof["attention_ms"] > 0 else 0.0
     tflops = flops_total / (call_ms * 1e-3) / 1e12 if call_ms > 0 else 0.0
-    tensor_bound = name == "C5"  # R = 2048 query rows per KV head: 580 flop per byte, above the ridge
+    tensor_bound = name.startswith("C5")  # R = 2048 query rows per KV head: 580 flop per byte, above the ridge
     ratio = NCU_TRAFFIC_RATIO.get(name) if args.kernel in (0, 2) else None
     roof = {"bound": "tensor" if tensor_bound else "hbm",
             "achieved": tflops if tensor_bound else achieved,
@@ -396,9 +403,12 @@ def measure_config(name, args, dev, peaks, sync, want_layer_modes, rank_world):
                        "q_heads": g.n_q_heads, "kv_heads": g.n_kv_heads, "head_dim": g.head_dim,
                        "decode_steps_in_schedule": wl.n_steps, "kv_cache_mb": cb.run.cache.numel() / 1e6,
                        "mb_streamed_per_step_min_mean_max": [round(x / 1e6, 1) for x in (
-                           min(wl.step_bytes(s)["total"] for s in range(wl.n_steps)),
-                           float(np.mean([wl.step_bytes(s)["total"] for s in range(wl.n_steps)])),
-                           max(wl.step_bytes(s)["total"] for s in range(wl.n_steps)))]}}
+                           min(wl.step_bytes(s, kvb)["total"] for s in range(wl.n_steps)),
+                           float(np.mean([wl.step_bytes(s, kvb)["total"] for s in range(wl.n_steps)])),
+                           max(wl.step_bytes(s, kvb)["total"] for s in range(wl.n_steps)))]}}
+    if kvb == 1:
+        entry["kv_cache"] = ("e4m3: rotated keys and values stored as 8-bit numbers; the byte figures count one byte per "
+                             "cache element, question-tokens/s compares directly with the bf16 entry of the workload")
     if want_layer_modes and args.kernel in (0, 2):
         entry["prefill"] = cb.prefill(peaks)
     if want_layer_modes:
@@ -488,6 +498,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-layer-modes", action="store_true", help="skip the per-layer launch modes and the prefill")
+    ap.add_argument("--kv-dtype", default="bf16", choices=["bf16", "e4m3"],
+                    help="cache element type of --config and of the --sweep table (a name in --also takes /e4m3)")
     ap.add_argument("--layers", type=int, default=0, help="override the number of layers (profiler captures)")
     ap.add_argument("--sweep", action="store_true",
                     help="questions-per-context x context-length table (the SWEEP-L*-Q* workloads) instead of the headline line")
@@ -520,7 +532,7 @@ def main():
     peaks = load_peaks()
     also = args.also
     if also is None:
-        also = ",".join(c for c in ("C2", "C3", "C5", "S1", "S2", "S3") if c != args.config) \
+        also = ",".join(c for c in ("C2", "C3", "C5", "S1", "S2", "S3", "C2/e4m3", "C3/e4m3") if c != args.config) \
             if (args.config == HEADLINE and world == 1) else ""
     others = [c for c in also.split(",") if c]
 
@@ -530,6 +542,7 @@ def main():
             dist.barrier()
             torch.cuda.synchronize()
 
+    kv_suffix = "/e4m3" if args.kv_dtype == "e4m3" else ""
     if args.sweep:
         # the axes of the paper's ablations: one JSON line holding the whole table
         from paper_2609_05707_b200 import workloads as W2
@@ -537,20 +550,20 @@ def main():
         rows = []
         for L in W2.SWEEP_CONTEXTS:
             for Q in W2.SWEEP_QUESTIONS:
-                e, c, _ = measure_config(f"SWEEP-L{L}-Q{Q}", args, dev, peaks, sync_all, False, 1)
+                e, c, _ = measure_config(f"SWEEP-L{L}-Q{Q}" + kv_suffix, args, dev, peaks, sync_all, False, 1)
                 c.close()
                 r = e["roofline"]
                 rows.append({"context": L, "questions": Q, "ms_per_step": e["ms_per_step"], "value": e["value"],
                              "call_us": r["avg_call_us"], "hbm_gbs": r["hbm_gbs"], "frac_of_8TBs": r["frac_of_8TBs"],
                              "frac": r["frac"], "read_probe_gbs": e["read_probe_gbs"]})
         if rank == 0:
-            print(json.dumps({"metric": METRIC, "unit": UNIT, "sweep": rows, "steps": args.steps, "warmup": args.warmup,
+            print(json.dumps({"metric": METRIC, "unit": UNIT, "kv_cache": args.kv_dtype, "sweep": rows, "steps": args.steps, "warmup": args.warmup,
                               "peak": peaks}), flush=True)
         return
 
     # ---- headline configuration ----
     t_wall0 = time.perf_counter()
-    entry, cb, (ms, tokens, timed, warm) = measure_config(args.config, args, dev, peaks, sync_all,
+    entry, cb, (ms, tokens, timed, warm) = measure_config(args.config + kv_suffix, args, dev, peaks, sync_all,
                                                           not args.no_layer_modes, 1)
     # headline figure: the timed region once more, clocks sampled while it runs
     sampler = ClockSampler(local_rank)
@@ -572,7 +585,7 @@ def main():
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         cpu = cpu_baseline(wl, 14.0)
 
-    per_config = {args.config: entry}
+    per_config = {args.config + kv_suffix: entry}
     for name in others:
         e, c, _ = measure_config(name, args, dev, peaks, sync_all, name == "C2" and not args.no_layer_modes, 1)
         c.close()
@@ -582,7 +595,8 @@ def main():
         sb = entry["shape"]["mb_streamed_per_step_min_mean_max"]
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": args.warmup, "ms_per_step": ms / len(timed), "higher_is_better": True, "scaling": "weak",
-                "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+                "vs_baseline": None, "dtype": "bf16" if not kv_suffix else "bf16 inputs and outputs, e4m3 cache",
+                "data": "synthetic",
                 "config": {"workload": wl.name, "prompts": wl.n_prompts, "questions": wl.n_questions,
                            "layers": g.n_layers, "q_heads": g.n_q_heads, "kv_heads": g.n_kv_heads,
                            "head_dim": g.head_dim, "decode_steps_in_schedule": wl.n_steps,

@@ -161,10 +161,11 @@ class Workload:
         return int(sum(len(self.active(s)) for s in range(self.n_steps)))
 
     # ---- algorithmic bytes / flops of one decode step over all layers ----
-    def step_bytes(self, s: int) -> Dict[str, int]:
+    def step_bytes(self, s: int, kv_elem_bytes: int = 2) -> Dict[str, int]:
+        """Algorithmic bytes of step s (all layers); kv_elem_bytes = 1 for the 8-bit cache variant."""
         g = self.geom
         act = self.active(s)
-        kvb = g.kv_bytes_per_token
+        kvb = g.kv_bytes_per_token * kv_elem_bytes // 2
         prompts = np.unique(self.prompt_of[act])
         # the shared instruction is read once for the whole batch, a context once per prompt with an active question
         ctx = (int(self.ctx_len[prompts].astype(np.int64).sum()) + (self.shared_len if len(act) else 0)) * kvb

@@ -37,11 +37,11 @@ def pick_stratified(wl, act, s, per_prompt):
     return out
 
 
-def run_and_sample(name, check, per_prompt, kernel=0, full_layer_step=None):
+def run_and_sample(name, check, per_prompt, kernel=0, full_layer_step=None, kv_dtype=B.KV_BF16):
     """check: {step: [(layer, kv head), ...]}.  Returns the number of tuples compared."""
     wl = W.make_workload(name)
     G = wl.geom.group
-    run = PoisonedRunner(wl, kernel=kernel)
+    run = PoisonedRunner(wl, kernel=kernel, kv_dtype=kv_dtype)
     run.load_header()
     # the K/V of every step go into the cache first (a token's slot depends only on its question and step index, and a
     # step reads no slot beyond its own), then only the sampled steps are run; each of them appends its own token again
@@ -55,7 +55,7 @@ def run_and_sample(name, check, per_prompt, kernel=0, full_layer_step=None):
         for layer, head in check[s]:
             everything = full_layer_step == (layer, s)
             qids = [int(k) for k in act] if everything else pick_stratified(wl, act, s, per_prompt)
-            ref = oracle_step(wl, s, layer, head, ctx_cache, step_cache, qids)
+            ref = oracle_step(wl, s, layer, head, ctx_cache, step_cache, qids, kv_e4m3=kv_dtype == B.KV_E4M3)
             o = out[layer, :, head * G:(head + 1) * G].float().cpu().numpy()
             got = np.stack([o[rows[k]] for k in qids])
             want = np.stack([ref[k] for k in qids])
@@ -102,6 +102,23 @@ def test_c3_full_size_sampled():
     lh = _layer_heads(wl, [(7, 5), (19, 2), (26, 6), (3, 3), (29, 1), (14, 7), (22, 0)])
     n = run_and_sample("C3", {s: lh for s in _steps(wl, [7, 40])}, per_prompt=32)
     assert n >= MIN_TUPLES, n
+
+
+def test_c2_full_size_sampled_e4m3_cache():
+    # the 8-bit cache variant in the bench's launch configuration, against the oracle over the quantised cache
+    wl = W.make_workload("C2")
+    lh = _layer_heads(wl, [(5, 1), (9, 6), (23, 2), (28, 5)])
+    check = {0: lh, 63: lh + [(17, h) for h in range(wl.geom.n_kv_heads)], 127: lh}
+    n = run_and_sample("C2", check, per_prompt=16, full_layer_step=(17, 63), kv_dtype=B.KV_E4M3)
+    assert n >= MIN_TUPLES // 2, n
+
+
+def test_c3_full_size_sampled_e4m3_cache():
+    wl = W.make_workload("C3")
+    lh = _layer_heads(wl, [(7, 5), (19, 2), (26, 6)])
+    last = int(wl.stop.max()) - 1
+    n = run_and_sample("C3", {s: lh for s in (0, 40, last)}, per_prompt=32, kv_dtype=B.KV_E4M3)
+    assert n >= 1024, n
 
 
 def test_c4_full_size_sampled():
