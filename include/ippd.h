@@ -147,7 +147,7 @@ int ippd_build_layout_shared(const ippd_geometry_t* geom, int32_t shared_len, in
 int ippd_layout_tables(const ippd_layout_t* layout, ippd_tables_t* out);
 
 /* Bytes and alignment of the K/V cache the caller must allocate on the device
- * (all layers; K and V; bf16).  Host-only. */
+ * (all layers; K and V; bf16, or one byte per element after IPPD_OPT_KV_DTYPE = IPPD_KV_E4M3).  Host-only. */
 int ippd_cache_bytes(const ippd_layout_t* layout, size_t* bytes, size_t* align);
 
 /*
