@@ -71,3 +71,17 @@ def test_sweep_and_shared_workloads_follow_their_recipes():
     # the instruction is counted once per step in the algorithmic bytes, every context once
     b = s3.step_bytes(0)
     assert b["context"] == (2754 + int(s3.ctx_len.sum())) * s3.geom.kv_bytes_per_token * 32
+
+
+def test_step_bytes_count_the_cache_by_its_element_size():
+    # algorithmic bytes of a step: the cache part halves on the 8-bit cache, queries and outputs stay bf16
+    wl = W.make_workload("C2")
+    g = wl.geom
+    for s in (0, 63, 127):
+        b2, b1 = wl.step_bytes(s), wl.step_bytes(s, 1)
+        assert b1["context"] * 2 == b2["context"] and b1["branch"] * 2 == b2["branch"]
+        assert b1["q_out"] == b2["q_out"] == len(wl.active(s)) * g.n_q_heads * g.head_dim * 2 * 2 * g.n_layers
+        assert b1["total"] == b1["context"] + b1["branch"] + b1["q_out"]
+        # by hand: one context of 2048 tokens, 16 branches of n_k + s + 1 tokens, K and V, 8 KV heads x 128 dims x 2 bytes
+        tokens = 2048 + int((wl.q_len[wl.active(s)] + s + 1).sum())
+        assert b2["context"] + b2["branch"] == tokens * 2 * g.n_kv_heads * g.head_dim * 2 * g.n_layers
