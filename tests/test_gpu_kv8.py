@@ -126,3 +126,35 @@ def test_the_cache_type_is_fixed_by_bind_and_needs_the_tensor_core_path():
         lay.set_option(B.OPT_KERNEL, 1)
     with pytest.raises(B.IppdError):
         lay.set_option(B.OPT_KV_DTYPE, 7)
+
+
+@pytest.mark.parametrize("tiles_per_split", [0, 3])
+def test_one_launch_step_equals_append_then_attention_bit_for_bit_e4m3(tiles_per_split):
+    # the fused append writes the same bytes as ippd_append_kv(STEP), and the attention then computes the same bits
+    from test_gpu_invariance import _base
+    base = _base()
+    res = []
+    for fused in (False, True):
+        run = PoisonedRunner(base, out_dtype=B.F32, tiles_per_split=tiles_per_split, fused=fused, layers_per_call=1,
+                             kv_dtype=B.KV_E4M3)
+        run.load_header()
+        outs = []
+        for s in range(base.n_steps):
+            act, out = run.run_step(s)
+            run.check()
+            outs.append(out.clone())
+        res.append((outs, run.cache.clone()))
+    for a, b in zip(res[0][0], res[1][0]):
+        assert torch.equal(a, b)
+    assert torch.equal(res[0][1], res[1][1])
+
+
+def test_question_order_does_not_change_an_answer_e4m3():
+    from test_gpu_invariance import Remapped, _all_steps, _base, _close
+    base = _base()
+    ref = _all_steps(base, kv_dtype=B.KV_E4M3)
+    r = np.random.default_rng(9)
+    perm = np.concatenate([lo + r.permutation(hi - lo) for lo, hi in zip(base.q_begin[:-1], base.q_begin[1:])])
+    got = _all_steps(Remapped.of(base, perm), kv_dtype=B.KV_E4M3)
+    for (j, s), o in got.items():
+        _close(o, ref[(int(perm[j]), s)], f"permuted question {j} step {s}, e4m3 cache")
